@@ -1,0 +1,183 @@
+/*
+ * peagle.h -- C ABI of the B200 (sm_100a) library for P-EAGLE's training-time drafter attention.
+ *
+ * The operation (paper Section 3, "Scalable Training Framework for Long Contexts"): every
+ * length-n sequence is expanded to K parallel-prediction depths, n*K tokens in all.  Token t
+ * carries (anchor[t], depth[t]); it sits at sequence position anchor+depth.  A query may attend
+ * to a key of the same sequence iff
+ *
+ *     (depth_k == 0 and anchor_k <= anchor_q)  or  (anchor_k == anchor_q and depth_k <= depth_q)
+ *
+ * i.e. the real context up to its anchor (Section 2: the depth-0 position is ordinary
+ * autoregressive prediction) plus its own chain at the same or earlier depths (Section 3: a
+ * depth-d position sees earlier depths only; Section 3.2: position p at depth d depends on
+ * position p-1 at depth d-1).  The library evaluates this predicate from the metadata inside
+ * its kernels; the (nK)^2 mask the paper pre-computes (Section 3.1) is never stored.
+ *
+ * Sequence partitioning (Section 3.2, Algorithm 1): attention runs one *query partition* at a
+ * time; a partition names its query rows and the keys those rows may see (its own segment plus
+ * the depth-0 tokens of earlier segments), and dK/dV are summed in fp32 over the partitions of
+ * a sequence (within-sequence gradient accumulation).
+ *
+ * Conventions for every entry point
+ *   - "dev" pointers are CUDA device pointers on the context's device, owned by the caller and
+ *     not retained after the call returns.  "host" pointers are ordinary host memory, read
+ *     before the call returns.
+ *   - Layouts (contiguous, base addresses 16-byte aligned):
+ *       Q, O, dO, dQ : bf16 [T][n_q_heads][head_dim]
+ *       K, V, dK, dV : bf16 [T][n_kv_heads][head_dim]
+ *       LSE          : fp32 [n_q_heads][T], natural-log log-sum-exp of the scaled scores
+ *       dK_acc,dV_acc: fp32 [T][n_kv_heads][head_dim]
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is enqueued on
+ *     it and the call returns without waiting, except where "synchronous" is stated.
+ *   - Return value: PEAGLE_OK (0) or a negative peagle_status.  Nothing aborts or throws.
+ *     Argument errors are detected on the host before anything is launched.  Errors found on
+ *     the device (bad metadata, a wait that ran out) are recorded in a status word that
+ *     peagle_poll_status() returns.
+ *   - A row whose visible allowed set is empty gets O = 0, LSE = -inf and zero gradients.
+ *   - Token order inside a sequence is free; only speed depends on it.
+ */
+#ifndef PEAGLE_H_
+#define PEAGLE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum peagle_status {
+    PEAGLE_OK = 0,
+    PEAGLE_ERR_NULL = -1,             /* a required pointer is NULL */
+    PEAGLE_ERR_BAD_SHAPE = -2,        /* head_dim not 64/128, heads not divisible, K out of [1,255], T mismatch */
+    PEAGLE_ERR_BAD_RANGE = -3,        /* range outside its sequence, unsorted or overlapping key ranges */
+    PEAGLE_ERR_BAD_META = -4,         /* depth outside [0,K) or anchor outside [0, 2^23) (device-side check) */
+    PEAGLE_ERR_UNSUPPORTED_ARCH = -5, /* device is not compute capability 10.x */
+    PEAGLE_ERR_WORKSPACE = -6,        /* scratch allocation failed */
+    PEAGLE_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired (device-side check) */
+    PEAGLE_ERR_TOO_LARGE = -8,        /* request exceeds a documented limit */
+    PEAGLE_ERR_CUDA = -9,             /* a CUDA runtime/driver call failed; see peagle_last_cuda_error */
+    PEAGLE_ERR_ALIGN = -10            /* a tensor base address is not 16-byte aligned */
+} peagle_status;
+
+typedef struct peagle_ctx peagle_ctx; /* opaque: device id, scratch memory, device status word */
+
+/* Half-open range of global token indices. */
+typedef struct peagle_range {
+    int32_t begin, end;
+} peagle_range_t;
+
+/* One batch of expanded sequences (Section 3: n x K positions per sequence). */
+typedef struct peagle_problem {
+    int32_t num_seqs;          /* >= 1 */
+    const int32_t *cu_seqlens; /* host [num_seqs+1]: expanded-token offsets, cu[0]=0, non-decreasing */
+    int32_t total_tokens;      /* T = cu_seqlens[num_seqs] */
+    const int32_t *anchor;     /* dev [T]: index (inside its sequence) of the last real token the chain starts from */
+    const int32_t *depth;      /* dev [T]: prediction depth, 0 <= depth < K */
+    int32_t K;                 /* number of depths, 1..255 */
+    int32_t n_q_heads, n_kv_heads, head_dim; /* n_q_heads % n_kv_heads == 0; head_dim 64 or 128 */
+    float softmax_scale;       /* usually 1/sqrt(head_dim) */
+} peagle_problem_t;
+
+/* One query partition of one sequence (Algorithm 1: a segment and the keys it may see). */
+typedef struct peagle_partition {
+    int32_t seq;             /* sequence index */
+    peagle_range_t q;        /* query rows, inside sequence `seq`; empty = no-op */
+    const peagle_range_t *k; /* host [nk]: visible keys, sorted disjoint non-empty ranges inside `seq` */
+    int32_t nk;              /* 0 = the whole sequence is visible */
+} peagle_partition_t;
+
+/* Creates a context on CUDA device `device` (sm_100 only).  Synchronous. */
+int peagle_create(peagle_ctx **out, int device);
+/* Frees the context and its scratch memory.  Synchronises the device first. */
+int peagle_destroy(peagle_ctx *ctx);
+const char *peagle_status_string(int status);
+/* Text of the last CUDA error the context saw (static storage inside the context). */
+const char *peagle_last_cuda_error(const peagle_ctx *ctx);
+/* Tile shape the kernels and peagle_classify_tiles use: BM query rows x BN keys. */
+int peagle_tile_shape(const peagle_ctx *ctx, int head_dim, int *BM, int *BN);
+/* Synchronises `stream`, returns and clears the device status word (PEAGLE_OK,
+ * PEAGLE_ERR_BAD_META or PEAGLE_ERR_TIMEOUT).  Synchronous. */
+int peagle_poll_status(peagle_ctx *ctx, void *stream);
+/* Number of kernels this library has launched through `ctx` since creation. */
+int64_t peagle_launch_count(const peagle_ctx *ctx);
+
+/*
+ * Forward of one query partition (Section 3; Algorithm 1 supplies the partition).
+ * For every row q in part->q, head h (kv head g = h / (n_q_heads/n_kv_heads)) and visible
+ * allowed key set A_q:   s_k = softmax_scale * <Q[q,h], K[k,g]>,
+ *   LSE[h][q] = log sum_{k in A_q} exp(s_k),   O[q,h] = sum_k exp(s_k - LSE) V[k,g].
+ * Writes O rows and LSE entries of the partition only.  All tensors dev.
+ */
+int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
+                    const void *Q, const void *K, const void *V, void *O, float *LSE, void *stream);
+
+/*
+ * Backward of one query partition (Section 3.2: one forward-backward per segment, gradients
+ * accumulated across the segments of a sequence).  With P = exp(s - LSE), Delta = <dO, O>,
+ * dP_k = <dO[q,h], V[k,g]>, dS_k = P_k (dP_k - Delta):
+ *   dQ[q,h]     = softmax_scale * sum_k dS_k K[k,g]              (rows of the partition, written)
+ *   dK_acc[k,g] += softmax_scale * sum_{q,h in group g} dS_k Q[q,h]   (ADDED)
+ *   dV_acc[k,g] += sum_{q,h in group g} P_k dO[q,h]                   (ADDED)
+ * The caller zeroes dK_acc/dV_acc once per sequence.  O and LSE are the forward's outputs for
+ * these rows.  Uses context scratch (fp32 dQ staging and Delta); concurrent calls on one
+ * context from different streams race.  All tensors dev.
+ */
+int peagle_attn_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
+                    const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                    const float *LSE, void *dQ, float *dK_acc, float *dV_acc, void *stream);
+
+/*
+ * The partition driver (Section 3.2 + Algorithm 1): zeroes internal fp32 dK/dV accumulators,
+ * then for each partition in the given order runs forward and backward (the partition's LSE is
+ * carried from its forward to its backward), and finally rounds the accumulated dK/dV to bf16.
+ * Every token of the batch should be a query in exactly one partition.  All tensors dev.
+ */
+int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
+                            const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                            const void *K, const void *V, const void *dO, void *O, float *LSE,
+                            void *dQ, void *dK, void *dV, void *stream);
+
+/*
+ * The same driver with HOST tensors: copies Q,K,V,dO and the metadata to the device, runs
+ * peagle_attn_partitioned, copies O, LSE, dQ, dK, dV back.  prob->anchor / prob->depth are HOST
+ * pointers for this call only.  Synchronous.  (Section 3.2; this is the end-to-end call.)
+ */
+int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
+                                 const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                                 const void *K, const void *V, const void *dO, void *O, float *LSE,
+                                 void *dQ, void *dK, void *dV);
+
+/*
+ * Algorithm 1, host only: segment of every token.  `boundaries` is host [S+1], context-token
+ * positions with boundaries[0]=0 and boundaries[S]=n (Algorithm 1's B).  Depth 0 and 1 tokens
+ * go by their position anchor+depth (a position at or beyond n stays in the last segment);
+ * deeper tokens inherit the segment of (anchor, depth-1).  anchor/depth/segment_out are host
+ * arrays over the `count` tokens of ONE sequence.  Returns PEAGLE_ERR_BAD_META if a token's
+ * dependency (anchor, depth-1) is absent.
+ */
+int peagle_assign_segments(const int32_t *anchor, const int32_t *depth, int32_t count, int32_t K,
+                           const int32_t *boundaries, int32_t S, int32_t *segment_out);
+
+/* ---- test hooks, synchronous ---- */
+
+/*
+ * Tile classes of one call (Section 3's mask, looked at BM x BN tiles): query tiles are BM rows
+ * from part->q.begin, key tiles BN tokens from the begin of each visible range.
+ * host_out[qt * n_ktiles + kt] = 0 SKIP (no allowed pair), 2 FULL (all BN keys present and every
+ * in-range row allows all of them), 1 PARTIAL.  host_out may be NULL to query the counts.
+ */
+int peagle_classify_tiles(peagle_ctx *ctx, const peagle_problem_t *prob,
+                          const peagle_partition_t *part, uint8_t *host_out, int32_t *n_qtiles,
+                          int32_t *n_ktiles);
+/*
+ * The mask of one call, materialised by the device predicate: host_out[(q - q.begin) * T + k]
+ * for every token k of the batch (1 = allowed and visible).  Only for q_len * T <= 2^26.
+ */
+int peagle_mask_dense(peagle_ctx *ctx, const peagle_problem_t *prob,
+                      const peagle_partition_t *part, uint8_t *host_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PEAGLE_H_ */

@@ -1,0 +1,618 @@
+// C ABI of libpeagle: context, argument validation, scratch memory, and the drivers that chain
+// K0 (mask evaluator / tile classifier / scheduler), K1 (forward) and K2 (backward).
+#include <stdio.h>
+#include <string.h>
+
+#include <vector>
+
+#include "peagle_internal.h"
+
+using namespace peagle;
+
+struct DevBuf {
+    void *ptr = nullptr;
+    size_t bytes = 0;
+};
+
+struct peagle_ctx {
+    int device = 0;
+    int n_sm = 0;
+    EncodeTiledFn encode = nullptr;
+    int *status = nullptr; // device status word
+    DevBuf plan_buf, bwd_buf, acc_buf, host_buf;
+    int64_t launches = 0;
+    char cuda_err[256] = {0};
+};
+
+namespace {
+
+int cuda_fail(peagle_ctx *ctx, cudaError_t e, const char *what)
+{
+    if (ctx)
+        snprintf(ctx->cuda_err, sizeof(ctx->cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return PEAGLE_ERR_CUDA;
+}
+
+#define CK(call)                                        \
+    do {                                                \
+        cudaError_t e_ = (call);                        \
+        if (e_ != cudaSuccess)                          \
+            return cuda_fail(ctx, e_, #call);           \
+    } while (0)
+
+// Grows a scratch buffer.  The old buffer may still be in use by work queued earlier, so the
+// stream is drained before it is freed.
+int ensure(peagle_ctx *ctx, DevBuf &b, size_t bytes, cudaStream_t s)
+{
+    if (bytes <= b.bytes)
+        return PEAGLE_OK;
+    if (b.ptr) {
+        CK(cudaStreamSynchronize(s));
+        CK(cudaFree(b.ptr));
+        b.ptr = nullptr;
+        b.bytes = 0;
+    }
+    const size_t want = bytes + bytes / 8 + 4096;
+    if (cudaMalloc(&b.ptr, want) != cudaSuccess) {
+        cudaGetLastError();
+        b.ptr = nullptr;
+        return PEAGLE_ERR_WORKSPACE;
+    }
+    b.bytes = want;
+    return PEAGLE_OK;
+}
+
+struct Carver {
+    uint8_t *base;
+    size_t off = 0;
+    explicit Carver(void *p) : base(static_cast<uint8_t *>(p)) {}
+    template <class T>
+    T *take(size_t n)
+    {
+        off = (off + 255) & ~size_t(255);
+        T *r = base ? reinterpret_cast<T *>(base + off) : nullptr;
+        off += n * sizeof(T);
+        return r;
+    }
+};
+
+void carve_plan(Plan &p, void *base, size_t *bytes_out)
+{
+    Carver c(base);
+    const size_t nq = (size_t)(p.n_qt > 0 ? p.n_qt : 1), nk = (size_t)(p.n_kt > 0 ? p.n_kt : 1);
+    p.meta = c.take<int32_t>((size_t)p.T);
+    p.ktile = c.take<int2>(nk);
+    p.qsum = c.take<int4>(nq);
+    p.ksum = c.take<int4>(nk);
+    p.cls = c.take<uint8_t>(nq * nk);
+    p.undecided = c.take<int>(nq * nk);
+    p.counters = c.take<int>(8);
+    p.klist = c.take<int2>(nq * nk);
+    p.kcount = c.take<int>(nq);
+    p.qorder = c.take<int>(nq);
+    p.qlist = c.take<int2>(nq * nk);
+    p.qcount = c.take<int>(nk);
+    p.bitems = c.take<int4>(nk * ((nq + BWD_CQ - 1) / BWD_CQ));
+    if (bytes_out)
+        *bytes_out = c.off + 256;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Call {
+    Plan plan;
+    RangeList ranges;
+    int seq_begin, seq_end;
+};
+
+int validate_problem(const peagle_problem_t *prob)
+{
+    if (!prob || !prob->cu_seqlens)
+        return PEAGLE_ERR_NULL;
+    if (prob->num_seqs < 1 || prob->total_tokens < 0)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (prob->head_dim != 64 && prob->head_dim != 128)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (prob->n_q_heads < 1 || prob->n_kv_heads < 1 || prob->n_q_heads % prob->n_kv_heads != 0)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (prob->K < 1 || prob->K > 255)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (!(prob->softmax_scale > 0.f))
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (prob->cu_seqlens[0] != 0 || prob->cu_seqlens[prob->num_seqs] != prob->total_tokens)
+        return PEAGLE_ERR_BAD_SHAPE;
+    for (int i = 0; i < prob->num_seqs; ++i)
+        if (prob->cu_seqlens[i + 1] < prob->cu_seqlens[i])
+            return PEAGLE_ERR_BAD_SHAPE;
+    if (prob->total_tokens > 0 && (!prob->anchor || !prob->depth))
+        return PEAGLE_ERR_NULL;
+    return PEAGLE_OK;
+}
+
+// Host-side checks of one partition; fills tile counts and the visible ranges.
+int validate_partition(const peagle_problem_t *prob, const peagle_partition_t *part, Call &c)
+{
+    if (!part)
+        return PEAGLE_ERR_NULL;
+    if (part->seq < 0 || part->seq >= prob->num_seqs)
+        return PEAGLE_ERR_BAD_RANGE;
+    const int sb = prob->cu_seqlens[part->seq], se = prob->cu_seqlens[part->seq + 1];
+    if (part->q.begin > part->q.end || part->q.begin < sb || part->q.end > se)
+        return PEAGLE_ERR_BAD_RANGE;
+    if (part->nk < 0 || (part->nk > 0 && !part->k))
+        return part->nk < 0 ? PEAGLE_ERR_BAD_RANGE : PEAGLE_ERR_NULL;
+    if (part->nk > MAX_KRANGES)
+        return PEAGLE_ERR_TOO_LARGE;
+    c.seq_begin = sb;
+    c.seq_end = se;
+    c.ranges.n = 0;
+    if (part->nk == 0) {
+        if (se > sb) {
+            c.ranges.n = 1;
+            c.ranges.begin[0] = sb;
+            c.ranges.end[0] = se;
+        }
+    } else {
+        int prev = sb;
+        for (int i = 0; i < part->nk; ++i) {
+            const peagle_range_t r = part->k[i];
+            if (r.begin >= r.end || r.begin < prev || r.end > se)
+                return PEAGLE_ERR_BAD_RANGE;
+            prev = r.end;
+            c.ranges.begin[i] = r.begin;
+            c.ranges.end[i] = r.end;
+        }
+        c.ranges.n = part->nk;
+    }
+    Plan &p = c.plan;
+    memset(&p, 0, sizeof(p));
+    p.T = prob->total_tokens;
+    p.q_begin = part->q.begin;
+    p.q_end = part->q.end;
+    p.n_qt = (p.q_end - p.q_begin + BM - 1) / BM;
+    p.n_kt = 0;
+    for (int i = 0; i < c.ranges.n; ++i)
+        p.n_kt += (c.ranges.end[i] - c.ranges.begin[i] + BN - 1) / BN;
+    return PEAGLE_OK;
+}
+
+// Runs K0 for one call.  On return c.plan points into ctx->plan_buf.
+int plan_call(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
+              bool for_bwd, cudaStream_t s, Call &c)
+{
+    int rc = validate_partition(prob, part, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    size_t bytes = 0;
+    carve_plan(c.plan, nullptr, &bytes);
+    rc = ensure(ctx, ctx->plan_buf, bytes, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    carve_plan(c.plan, ctx->plan_buf.ptr, nullptr);
+    c.plan.status = ctx->status;
+    if (c.plan.n_qt == 0)
+        return PEAGLE_OK;
+    ctx->launches += launch_plan(c.plan, prob->anchor, prob->depth, prob->K, c.seq_begin, c.seq_end,
+                                 c.ranges, for_bwd, prob->n_kv_heads, s);
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int run_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const void *Q,
+            const void *K, const void *V, void *O, float *LSE, cudaStream_t s)
+{
+    if (c.plan.n_qt == 0)
+        return PEAGLE_OK;
+    FwdArgs a;
+    a.Q = Q;
+    a.K = K;
+    a.V = V;
+    a.O = O;
+    a.LSE = LSE;
+    a.Hq = prob->n_q_heads;
+    a.Hkv = prob->n_kv_heads;
+    a.D = prob->head_dim;
+    a.scale = prob->softmax_scale;
+    const int n = launch_fwd(c.plan, a, ctx->encode, ctx->n_sm, s);
+    if (n < 0)
+        return n;
+    ctx->launches += n;
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const void *Q,
+            const void *K, const void *V, const void *O, const void *dO, const float *LSE,
+            void *dQ, float *dK_acc, float *dV_acc, cudaStream_t s)
+{
+    if (c.plan.n_qt == 0)
+        return PEAGLE_OK;
+    const size_t q_len = (size_t)(c.plan.q_end - c.plan.q_begin);
+    const size_t Hq = (size_t)prob->n_q_heads, D = (size_t)prob->head_dim;
+    const size_t delta_bytes = ((Hq * q_len * 4 + 255) / 256) * 256;
+    const size_t dq_bytes = q_len * Hq * D * 4;
+    int rc = ensure(ctx, ctx->bwd_buf, delta_bytes + dq_bytes + 256, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    BwdArgs a;
+    a.Q = Q;
+    a.K = K;
+    a.V = V;
+    a.O = O;
+    a.dO = dO;
+    a.LSE = LSE;
+    a.dQ = dQ;
+    a.dK_acc = dK_acc;
+    a.dV_acc = dV_acc;
+    a.delta = static_cast<float *>(ctx->bwd_buf.ptr);
+    a.dq_acc = reinterpret_cast<float *>(static_cast<uint8_t *>(ctx->bwd_buf.ptr) + delta_bytes);
+    a.Hq = prob->n_q_heads;
+    a.Hkv = prob->n_kv_heads;
+    a.D = prob->head_dim;
+    a.scale = prob->softmax_scale;
+    const int n = launch_bwd(c.plan, a, ctx->encode, ctx->n_sm, s);
+    if (n < 0)
+        return n;
+    ctx->launches += n;
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int peagle_create(peagle_ctx **out, int device)
+{
+    if (!out)
+        return PEAGLE_ERR_NULL;
+    *out = nullptr;
+    peagle_ctx *ctx = new peagle_ctx();
+    ctx->device = device;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaSetDevice(device);
+    if (e == cudaSuccess)
+        e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) {
+        delete ctx;
+        return PEAGLE_ERR_CUDA;
+    }
+    if (prop.major != 10) {
+        delete ctx;
+        return PEAGLE_ERR_UNSUPPORTED_ARCH;
+    }
+    ctx->n_sm = prop.multiProcessorCount;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        delete ctx;
+        return PEAGLE_ERR_CUDA;
+    }
+    ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    if (cudaMalloc(&ctx->status, 256) != cudaSuccess || cudaMemset(ctx->status, 0, 256) != cudaSuccess) {
+        delete ctx;
+        return PEAGLE_ERR_WORKSPACE;
+    }
+    *out = ctx;
+    return PEAGLE_OK;
+}
+
+int peagle_destroy(peagle_ctx *ctx)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    DevBuf *bufs[4] = {&ctx->plan_buf, &ctx->bwd_buf, &ctx->acc_buf, &ctx->host_buf};
+    for (DevBuf *b : bufs)
+        if (b->ptr)
+            cudaFree(b->ptr);
+    if (ctx->status)
+        cudaFree(ctx->status);
+    delete ctx;
+    return PEAGLE_OK;
+}
+
+const char *peagle_status_string(int status)
+{
+    switch (status) {
+    case PEAGLE_OK: return "ok";
+    case PEAGLE_ERR_NULL: return "null pointer";
+    case PEAGLE_ERR_BAD_SHAPE: return "bad shape";
+    case PEAGLE_ERR_BAD_RANGE: return "bad range";
+    case PEAGLE_ERR_BAD_META: return "bad token metadata";
+    case PEAGLE_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    case PEAGLE_ERR_WORKSPACE: return "scratch allocation failed";
+    case PEAGLE_ERR_TIMEOUT: return "device-side wait timed out";
+    case PEAGLE_ERR_TOO_LARGE: return "request exceeds a limit";
+    case PEAGLE_ERR_CUDA: return "CUDA error";
+    case PEAGLE_ERR_ALIGN: return "tensor not 16-byte aligned";
+    default: return "unknown status";
+    }
+}
+
+const char *peagle_last_cuda_error(const peagle_ctx *ctx) { return ctx ? ctx->cuda_err : ""; }
+
+int peagle_tile_shape(const peagle_ctx *ctx, int head_dim, int *bm, int *bn)
+{
+    (void)ctx;
+    if (!bm || !bn)
+        return PEAGLE_ERR_NULL;
+    if (head_dim != 64 && head_dim != 128)
+        return PEAGLE_ERR_BAD_SHAPE;
+    *bm = BM;
+    *bn = BN;
+    return PEAGLE_OK;
+}
+
+int peagle_poll_status(peagle_ctx *ctx, void *stream)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st = 0;
+    CK(cudaStreamSynchronize(s));
+    CK(cudaMemcpy(&st, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (st != 0)
+        CK(cudaMemset(ctx->status, 0, sizeof(int)));
+    return st;
+}
+
+int64_t peagle_launch_count(const peagle_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
+                    const void *Q, const void *K, const void *V, void *O, float *LSE, void *stream)
+{
+    if (!ctx || !Q || !K || !V || !O || !LSE)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))
+        return PEAGLE_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CK(cudaSetDevice(ctx->device));
+    Call c;
+    rc = plan_call(ctx, prob, part, false, s, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    return run_fwd(ctx, prob, c, Q, K, V, O, LSE, s);
+}
+
+int peagle_attn_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
+                    const void *Q, const void *K, const void *V, const void *O, const void *dO,
+                    const float *LSE, void *dQ, float *dK_acc, float *dV_acc, void *stream)
+{
+    if (!ctx || !Q || !K || !V || !O || !dO || !LSE || !dQ || !dK_acc || !dV_acc)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK_acc) || !aligned16(dV_acc))
+        return PEAGLE_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CK(cudaSetDevice(ctx->device));
+    Call c;
+    rc = plan_call(ctx, prob, part, true, s, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    return run_bwd(ctx, prob, c, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc, s);
+}
+
+int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
+                            const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                            const void *K, const void *V, const void *dO, void *O, float *LSE,
+                            void *dQ, void *dK, void *dV, void *stream)
+{
+    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV || (nparts > 0 && !parts))
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (nparts < 0)
+        return PEAGLE_ERR_BAD_RANGE;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return PEAGLE_ERR_ALIGN;
+    {   // check every partition before anything is launched
+        Call tmp;
+        for (int i = 0; i < nparts; ++i) {
+            rc = validate_partition(prob, &parts[i], tmp);
+            if (rc != PEAGLE_OK)
+                return rc;
+        }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CK(cudaSetDevice(ctx->device));
+    const size_t n_kv = (size_t)prob->total_tokens * prob->n_kv_heads * prob->head_dim;
+    if (n_kv == 0)
+        return PEAGLE_OK;
+    rc = ensure(ctx, ctx->acc_buf, 2 * n_kv * sizeof(float), s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    float *dK_acc = static_cast<float *>(ctx->acc_buf.ptr);
+    float *dV_acc = dK_acc + n_kv;
+    CK(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s));
+    for (int i = 0; i < nparts; ++i) {
+        Call c;
+        rc = plan_call(ctx, prob, &parts[i], true, s, c);
+        if (rc != PEAGLE_OK)
+            return rc;
+        rc = run_fwd(ctx, prob, c, Q, K, V, O, LSE, s);
+        if (rc != PEAGLE_OK)
+            return rc;
+        rc = run_bwd(ctx, prob, c, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc, s);
+        if (rc != PEAGLE_OK)
+            return rc;
+    }
+    ctx->launches += launch_cast_grads(dK_acc, dV_acc, dK, dV, n_kv, s);
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
+                                 const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                                 const void *K, const void *V, const void *dO, void *O, float *LSE,
+                                 void *dQ, void *dK, void *dV)
+{
+    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t s = nullptr;
+    const size_t T = (size_t)prob->total_tokens;
+    const size_t nq = T * prob->n_q_heads * prob->head_dim * 2;  // bytes of a bf16 query-side tensor
+    const size_t nkv = T * prob->n_kv_heads * prob->head_dim * 2;
+    const size_t nlse = T * prob->n_q_heads * 4;
+    const size_t nmeta = T * 4;
+    auto up = [](size_t b) { return (b + 255) & ~size_t(255); };
+    const size_t total = 4 * up(nq) + 4 * up(nkv) + up(nlse) + 2 * up(nmeta) + 256;
+    rc = ensure(ctx, ctx->host_buf, total, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    uint8_t *b = static_cast<uint8_t *>(ctx->host_buf.ptr);
+    uint8_t *dQin = b;            b += up(nq);
+    uint8_t *ddO = b;             b += up(nq);
+    uint8_t *dOout = b;           b += up(nq);
+    uint8_t *ddQ = b;             b += up(nq);
+    uint8_t *dKin = b;            b += up(nkv);
+    uint8_t *dVin = b;            b += up(nkv);
+    uint8_t *ddK = b;             b += up(nkv);
+    uint8_t *ddV = b;             b += up(nkv);
+    uint8_t *dLSE = b;            b += up(nlse);
+    uint8_t *danchor = b;         b += up(nmeta);
+    uint8_t *ddepth = b;
+    CK(cudaMemcpyAsync(dQin, Q, nq, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(dKin, K, nkv, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(dVin, V, nkv, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(ddO, dO, nq, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(danchor, prob->anchor, nmeta, cudaMemcpyHostToDevice, s));
+    CK(cudaMemcpyAsync(ddepth, prob->depth, nmeta, cudaMemcpyHostToDevice, s));
+    peagle_problem_t dprob = *prob;
+    dprob.anchor = reinterpret_cast<const int32_t *>(danchor);
+    dprob.depth = reinterpret_cast<const int32_t *>(ddepth);
+    rc = peagle_attn_partitioned(ctx, &dprob, parts, nparts, dQin, dKin, dVin, ddO, dOout,
+                                 reinterpret_cast<float *>(dLSE), ddQ, ddK, ddV, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    CK(cudaMemcpyAsync(O, dOout, nq, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(LSE, dLSE, nlse, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(dQ, ddQ, nq, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(dK, ddK, nkv, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemcpyAsync(dV, ddV, nkv, cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    return PEAGLE_OK;
+}
+
+int peagle_assign_segments(const int32_t *anchor, const int32_t *depth, int32_t count, int32_t K,
+                           const int32_t *boundaries, int32_t S, int32_t *segment_out)
+{
+    if (!anchor || !depth || !boundaries || !segment_out)
+        return PEAGLE_ERR_NULL;
+    if (S < 1 || K < 1 || count < 0)
+        return PEAGLE_ERR_BAD_SHAPE;
+    const int n = boundaries[S];
+    if (boundaries[0] != 0 || n < 0)
+        return PEAGLE_ERR_BAD_RANGE;
+    for (int s = 0; s < S; ++s)
+        if (boundaries[s + 1] < boundaries[s])
+            return PEAGLE_ERR_BAD_RANGE;
+    // seg_of[d][a] for the tokens present, -1 elsewhere; filled depth by depth.
+    std::vector<std::vector<int32_t>> seg_of((size_t)K, std::vector<int32_t>((size_t)n, -1));
+    for (int i = 0; i < count; ++i)
+        if (depth[i] < 0 || depth[i] >= K || anchor[i] < 0 || anchor[i] >= n)
+            return PEAGLE_ERR_BAD_META;
+    auto by_position = [&](int pos) {
+        int s = 0;
+        while (s + 1 <= S && boundaries[s + 1] <= pos)
+            ++s; // largest s with boundaries[s] <= pos
+        return s < S ? s : S - 1;
+    };
+    for (int d = 0; d < K; ++d)
+        for (int i = 0; i < count; ++i) {
+            if (depth[i] != d)
+                continue;
+            int s;
+            if (d <= 1) {
+                s = by_position(anchor[i] + d);
+            } else {
+                s = seg_of[(size_t)d - 1][(size_t)anchor[i]];
+                if (s < 0)
+                    return PEAGLE_ERR_BAD_META;
+            }
+            seg_of[(size_t)d][(size_t)anchor[i]] = s;
+            segment_out[i] = s;
+        }
+    return PEAGLE_OK;
+}
+
+int peagle_classify_tiles(peagle_ctx *ctx, const peagle_problem_t *prob,
+                          const peagle_partition_t *part, uint8_t *host_out, int32_t *n_qtiles,
+                          int32_t *n_ktiles)
+{
+    if (!ctx || !n_qtiles || !n_ktiles)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    CK(cudaSetDevice(ctx->device));
+    Call c;
+    if (!host_out) {
+        rc = validate_partition(prob, part, c);
+        if (rc != PEAGLE_OK)
+            return rc;
+        *n_qtiles = c.plan.n_qt;
+        *n_ktiles = c.plan.n_kt;
+        return PEAGLE_OK;
+    }
+    rc = plan_call(ctx, prob, part, true, nullptr, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    *n_qtiles = c.plan.n_qt;
+    *n_ktiles = c.plan.n_kt;
+    CK(cudaStreamSynchronize(nullptr));
+    if (c.plan.n_qt > 0 && c.plan.n_kt > 0)
+        CK(cudaMemcpy(host_out, c.plan.cls, (size_t)c.plan.n_qt * c.plan.n_kt, cudaMemcpyDeviceToHost));
+    return PEAGLE_OK;
+}
+
+int peagle_mask_dense(peagle_ctx *ctx, const peagle_problem_t *prob,
+                      const peagle_partition_t *part, uint8_t *host_out)
+{
+    if (!ctx || !host_out)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    CK(cudaSetDevice(ctx->device));
+    Call c;
+    rc = validate_partition(prob, part, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    const size_t q_len = (size_t)(c.plan.q_end - c.plan.q_begin);
+    const size_t n = q_len * (size_t)c.plan.T;
+    if (n > (size_t(1) << 26))
+        return PEAGLE_ERR_TOO_LARGE;
+    if (n == 0)
+        return PEAGLE_OK;
+    rc = plan_call(ctx, prob, part, false, nullptr, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    uint8_t *dev = nullptr;
+    if (cudaMalloc(&dev, n) != cudaSuccess) {
+        cudaGetLastError();
+        return PEAGLE_ERR_WORKSPACE;
+    }
+    ctx->launches += launch_mask_dense(c.plan, c.ranges, dev, nullptr);
+    cudaError_t e = cudaMemcpy(host_out, dev, n, cudaMemcpyDeviceToHost);
+    cudaFree(dev);
+    if (e != cudaSuccess)
+        return cuda_fail(ctx, e, "cudaMemcpy(mask)");
+    return PEAGLE_OK;
+}
+
+} // extern "C"

@@ -1,0 +1,428 @@
+// K1: forward of one query partition on sm_100a.
+//
+// One CTA owns one query tile (128 rows) for two query heads of the same KV group (or one head
+// when the group size is odd), so both tiles share the K/V tiles staged in shared memory and the
+// same mask.  Roles:
+//   warps 0-3  softmax of tile A (one query row per thread; online softmax in the log2 domain,
+//              log-sum-exp bookkeeping, final normalisation and store)
+//   warps 4-7  softmax of tile B
+//   warp  8    allocates tensor memory; lane 0 issues every tcgen05.mma
+//   warp  9    producer: TMA loads of Q once and of the K / V tiles through a ring, plus the
+//              packed metadata of each key tile for the implicit mask
+// Tensor memory (512 columns x 128 lanes, fp32): S_A | S_B (128 columns each; the bf16
+// probabilities overwrite the first 64 columns of their own S), then O_A | O_B (head_dim each).
+// S = Q K^T takes both operands from shared memory (K-major, 128-byte swizzle); O += P V takes
+// P from tensor memory and V from shared memory (MN-major).  The MMA thread interleaves the two
+// tiles so that the tensor cores work on one while the other is in its softmax.
+// Only tiles the classifier kept are visited; FULL tiles skip the per-element predicate.
+#include <math_constants.h>
+
+#include "peagle_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace peagle {
+using namespace sm100;
+
+struct FwdParams {
+    const int2 *klist;
+    const int *kcount;
+    const int *qorder;
+    const int32_t *meta;
+    int *status;
+    int n_kt, q_begin, q_end, T;
+    __nv_bfloat16 *O;
+    float *LSE;
+    int Hq, Hkv;
+    int two; // 1: two heads per CTA
+    float scale_log2;
+};
+
+template <int D>
+struct FwdCfg {
+    static constexpr int NS = (D == 64) ? 3 : 2;
+    static constexpr int PANELS = D / 64;
+    static constexpr int PANEL_BYTES = 128 * 128; // 128 rows of 128 bytes
+    static constexpr int TILE_BYTES = PANELS * PANEL_BYTES;
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_K = 2 * TILE_BYTES;
+    static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
+    static constexpr int OFF_META = OFF_V + NS * TILE_BYTES;
+    static constexpr int OFF_BAR = OFF_META + NS * BN * 4;
+    static constexpr int N_BAR = 1 + 4 * NS + 6;
+    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
+    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024; // + slack for 1024-byte alignment
+    static constexpr int TM_S = 0;      // S_A at 0, S_B at 128
+    static constexpr int TM_O = 256;    // O_A at 256, O_B at 256 + D
+};
+
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+           const __grid_constant__ CUtensorMap tmV, const FwdParams P)
+{
+    using C = FwdCfg<D>;
+    constexpr int NS = C::NS;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u;
+    uint8_t *sp = smem_raw + (sb - raw);
+
+    const uint32_t bar0 = sb + C::OFF_BAR;
+    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    // barrier indices
+    constexpr int B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 1 + NS, B_VFULL = 1 + 2 * NS,
+                  B_VEMPTY = 1 + 3 * NS, B_SFULL = 1 + 4 * NS, B_PFULL = B_SFULL + 2,
+                  B_ODONE = B_SFULL + 4;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
+    int32_t *smeta = reinterpret_cast<int32_t *>(sp + C::OFF_META);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ntile = P.two ? 2 : 1;
+    const int n_hb = P.two ? P.Hq / 2 : P.Hq;
+    const int qt = P.qorder[blockIdx.x / n_hb];
+    const int hb = blockIdx.x % n_hb;
+    const int h0 = P.two ? 2 * hb : hb;
+    const int g = h0 / (P.Hq / P.Hkv);
+    const int row0 = P.q_begin + qt * BM;
+    const int cnt = P.kcount[qt];
+    const int2 *klist = P.klist + (size_t)qt * P.n_kt;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        mbar_init(BAR(B_QFULL), 1);
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(BAR(B_KFULL + s), 1);
+            mbar_init(BAR(B_KEMPTY + s), 1);
+            mbar_init(BAR(B_VFULL + s), 1);
+            mbar_init(BAR(B_VEMPTY + s), 1);
+        }
+        for (int x = 0; x < 2; ++x) {
+            mbar_init(BAR(B_SFULL + x), 1);
+            mbar_init(BAR(B_PFULL + x), 128);
+            mbar_init(BAR(B_ODONE + x), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(sb + C::OFF_MISC, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 9) {
+        // ------------------------------------------------------------ producer
+        if (cnt > 0) {
+            if (lane == 0) {
+                tma_prefetch_desc(&tmQ);
+                tma_prefetch_desc(&tmK);
+                tma_prefetch_desc(&tmV);
+                mbar_arrive_expect_tx(BAR(B_QFULL), ntile * C::TILE_BYTES);
+                for (int x = 0; x < ntile; ++x)
+                    for (int pn = 0; pn < C::PANELS; ++pn)
+                        tma_load_3d(sb + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmQ,
+                                    BAR(B_QFULL), pn * 64, h0 + x, row0);
+            }
+            for (int j = 0; j < cnt; ++j) {
+                const int st = j % NS, ph = (j / NS) & 1;
+                const int2 e = klist[j];
+                const int start = e.x, len = e.y & 0xffff;
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(BAR(B_KEMPTY + st), ph ^ 1, abort_flag);
+                    if (ok) {
+                        mbar_arrive_expect_tx(BAR(B_KFULL + st), C::TILE_BYTES);
+                        for (int pn = 0; pn < C::PANELS; ++pn)
+                            tma_load_3d(sb + C::OFF_K + st * C::TILE_BYTES + pn * C::PANEL_BYTES,
+                                        &tmK, BAR(B_KFULL + st), pn * 64, g, start);
+                    }
+                }
+                ok = ok && mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, abort_flag);
+                if (!__all_sync(0xffffffffu, ok))
+                    break;
+                for (int i = lane; i < BN; i += 32)
+                    smeta[st * BN + i] = (i < len) ? P.meta[start + i] : META_NONE_K;
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(BAR(B_VFULL + st), C::TILE_BYTES);
+                    for (int pn = 0; pn < C::PANELS; ++pn)
+                        tma_load_3d(sb + C::OFF_V + st * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmV,
+                                    BAR(B_VFULL + st), pn * 64, g, start);
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0 && cnt > 0) {
+            constexpr uint32_t IDESC_S = idesc_bf16_f32(128, BN, 0, 0);
+            constexpr uint32_t IDESC_O = idesc_bf16_f32(128, D, 0, 1);
+            auto issue_s = [&](int x, int st) {
+                const uint32_t qa = sb + C::OFF_Q + x * C::TILE_BYTES;
+                const uint32_t ka = sb + C::OFF_K + st * C::TILE_BYTES;
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k) {
+                    const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
+                    mma_ss(tmem + C::TM_S + x * 128, smem_desc_sw128(qa + off, 16, 1024),
+                           smem_desc_sw128(ka + off, 16, 1024), IDESC_S, k > 0);
+                }
+            };
+            auto issue_pv = [&](int x, int st, bool acc) {
+                const uint32_t va = sb + C::OFF_V + st * C::TILE_BYTES;
+#pragma unroll
+                for (int k = 0; k < BN / 16; ++k)
+                    mma_ts(tmem + C::TM_O + x * D, tmem + C::TM_S + x * 128 + k * 8,
+                           smem_desc_sw128(va + k * 2048, C::PANEL_BYTES, 1024), IDESC_O,
+                           acc || k > 0);
+            };
+            bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag) &&
+                      mbar_wait(BAR(B_KFULL + 0), 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                for (int x = 0; x < ntile; ++x) {
+                    issue_s(x, 0);
+                    tc_commit(BAR(B_SFULL + x));
+                }
+                tc_commit(BAR(B_KEMPTY + 0));
+            }
+            for (int j = 0; ok && j < cnt; ++j) {
+                const int st = j % NS, ph = (j / NS) & 1;
+                const int nst = (j + 1) % NS, nph = ((j + 1) / NS) & 1;
+                const bool more = j + 1 < cnt;
+                ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
+                if (ok && more)
+                    ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag);
+                for (int x = 0; ok && x < ntile; ++x) {
+                    ok = mbar_wait(BAR(B_PFULL + x), j & 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    issue_pv(x, st, j > 0);
+                    if (x == ntile - 1)
+                        tc_commit(BAR(B_VEMPTY + st));
+                    if (more) {
+                        issue_s(x, nst);
+                        tc_commit(BAR(B_SFULL + x));
+                        if (x == ntile - 1)
+                            tc_commit(BAR(B_KEMPTY + nst));
+                    } else {
+                        tc_commit(BAR(B_ODONE + x));
+                    }
+                }
+            }
+        }
+    } else if (warp < 4 * ntile) {
+        // ------------------------------------------------------------ softmax of tile x
+        const int x = warp >> 2;
+        const int r = threadIdx.x & 127;
+        const int h = h0 + x;
+        const int row = row0 + r;
+        const bool row_ok = row < P.q_end;
+        int32_t mq = row_ok ? P.meta[row] : META_NONE_Q;
+        if (mq == META_NONE_K)
+            mq = META_NONE_Q;
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_sel + C::TM_S + x * 128;
+        const uint32_t tO = tmem + lane_sel + C::TM_O + x * D;
+        float m = -CUDART_INF_F, l = 0.f;
+        bool ok = true;
+        for (int j = 0; j < cnt; ++j) {
+            const int st = j % NS, ph = (j / NS) & 1;
+            const int cls = klist[j].y >> 16;
+            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL + x), j & 1, abort_flag));
+            if (!ok)
+                break;
+            tc_fence_after();
+            uint32_t xr[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                tmem_ld32(tS + c * 32, xr[c]);
+            tmem_wait_ld();
+            if (cls != TILE_FULL) {
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
+                if (!ok)
+                    break;
+                const int4 *mk4 = reinterpret_cast<const int4 *>(smeta + st * BN);
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        const int4 mk = mk4[(c * 32 + i) >> 2];
+                        if (!allowed_packed(mq, mk.x)) xr[c][i + 0] = 0xff800000u;
+                        if (!allowed_packed(mq, mk.y)) xr[c][i + 1] = 0xff800000u;
+                        if (!allowed_packed(mq, mk.z)) xr[c][i + 2] = 0xff800000u;
+                        if (!allowed_packed(mq, mk.w)) xr[c][i + 3] = 0xff800000u;
+                    }
+            }
+            float mx = -CUDART_INF_F;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    mx = fmaxf(mx, __uint_as_float(xr[c][i]));
+            mx *= P.scale_log2; // scale > 0, so the max commutes with the scaling
+            const float m_new = fmaxf(m, mx);
+            if (j == 0) {
+                m = m_new;
+            } else {
+                // Rescale the running output only when the maximum grew by more than 2^8; until
+                // then the stale maximum keeps every probability below 256.
+                const bool grow = m_new > m + 8.f;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float alpha = (m_new == -CUDART_INF_F) ? 1.f : fast_exp2(m - m_new);
+                    l *= alpha;
+                    m = m_new;
+#pragma unroll
+                    for (int c = 0; c < D / 32; ++c) {
+                        uint32_t o[32];
+                        tmem_ld32(tO + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            o[i] = __float_as_uint(__uint_as_float(o[i]) * alpha);
+                        tmem_st32(tO + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            const float neg_m = (m == -CUDART_INF_F) ? 0.f : -m;
+            float sum = 0.f;
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const int c0 = 2 * i + 64 * c; // columns c0, c0+1 of this row
+                    const float p0 = fast_exp2(fmaf(__uint_as_float(xr[c0 >> 5][c0 & 31]),
+                                                    P.scale_log2, neg_m));
+                    const float p1 = fast_exp2(fmaf(__uint_as_float(xr[(c0 + 1) >> 5][(c0 + 1) & 31]),
+                                                    P.scale_log2, neg_m));
+                    sum += p0 + p1;
+                    pk[i] = pack_bf16x2(p0, p1);
+                }
+                tmem_st32(tS + c * 32, pk);
+            }
+            l += sum;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(BAR(B_PFULL + x));
+        }
+        // ---- epilogue: normalise, store O and LSE
+        if (cnt == 0) {
+            if (row_ok) {
+                uint4 z = make_uint4(0, 0, 0, 0);
+                uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
+                for (int i = 0; i < D / 8; ++i)
+                    dst[i] = z;
+                P.LSE[(size_t)h * P.T + row] = -CUDART_INF_F;
+            }
+        } else if (__all_sync(0xffffffffu, ok && mbar_wait(BAR(B_ODONE + x), 0, abort_flag))) {
+            tc_fence_after();
+            const float inv = l > 0.f ? 1.f / l : 0.f;
+            uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(tO + c * 32, o);
+                tmem_wait_ld();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                        dst[c * 4 + (i >> 3)] = v;
+                    }
+                }
+            }
+            if (row_ok)
+                P.LSE[(size_t)h * P.T + row] =
+                    l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
+        }
+    }
+
+    // ------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
+        // give copies and MMAs that may still be in flight time to land before the CTA's
+        // shared and tensor memory are released
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {
+        }
+        __syncthreads();
+    }
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+static int make_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int H, int T)
+{
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)T};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)H * D * 2};
+    cuuint32_t box[3] = {64, 1, 128};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides,
+                     box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? 0 : -1;
+}
+
+int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int H, int T)
+{
+    return make_map(enc, m, base, D, H, T);
+}
+
+template <int D>
+static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cudaStream_t s)
+{
+    CUtensorMap tmQ, tmK, tmV;
+    if (make_map(enc, &tmQ, a.Q, D, a.Hq, p.T) || make_map(enc, &tmK, a.K, D, a.Hkv, p.T) ||
+        make_map(enc, &tmV, a.V, D, a.Hkv, p.T))
+        return PEAGLE_ERR_CUDA;
+    FwdParams P;
+    P.klist = p.klist;
+    P.kcount = p.kcount;
+    P.qorder = p.qorder;
+    P.meta = p.meta;
+    P.status = p.status;
+    P.n_kt = p.n_kt;
+    P.q_begin = p.q_begin;
+    P.q_end = p.q_end;
+    P.T = p.T;
+    P.O = static_cast<__nv_bfloat16 *>(a.O);
+    P.LSE = a.LSE;
+    P.Hq = a.Hq;
+    P.Hkv = a.Hkv;
+    P.two = ((a.Hq / a.Hkv) % 2 == 0) ? 1 : 0;
+    P.scale_log2 = a.scale * 1.4426950408889634f;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 FwdCfg<D>::SMEM_BYTES) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        attr_set = true;
+    }
+    const int n_hb = P.two ? a.Hq / 2 : a.Hq;
+    fwd_kernel<D><<<p.n_qt * n_hb, 320, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
+    return 1;
+}
+
+int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+{
+    (void)n_sm;
+    if (p.n_qt == 0)
+        return 0;
+    return a.D == 64 ? launch_fwd_t<64>(p, a, enc, s) : launch_fwd_t<128>(p, a, enc, s);
+}
+
+} // namespace peagle

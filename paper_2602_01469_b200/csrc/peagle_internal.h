@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of libpeagle.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/peagle.h"
+
+namespace peagle {
+
+constexpr int BM = 128;          // query rows per tile
+constexpr int BN = 128;          // keys per tile
+constexpr int MAX_KRANGES = 32;  // visible key ranges per partition
+constexpr int BWD_CQ = 8;        // query tiles per backward work item
+constexpr int32_t META_NONE_Q = -1;         // packed metadata of a row outside the partition (sees nothing)
+constexpr int32_t META_NONE_K = 0x7fffffff; // packed metadata of a key outside the batch (seen by nobody)
+
+enum TileClass : uint8_t { TILE_SKIP = 0, TILE_PARTIAL = 1, TILE_FULL = 2 };
+
+// Visible key ranges of one call, passed to kernels by value.
+struct RangeList {
+    int n;
+    int begin[MAX_KRANGES];
+    int end[MAX_KRANGES];
+};
+
+// Everything the mask evaluator / tile classifier / scheduler (K0) produces for one call.
+// All pointers are device memory inside the context's scratch buffer.
+struct Plan {
+    int T;                 // tokens in the batch
+    int q_begin, q_end;    // query rows of the call
+    int n_qt, n_kt;        // tile counts
+    int32_t *meta;         // [T] packed (anchor << 8 | depth)
+    int2 *ktile;           // [n_kt] (first token, length)
+    int4 *qsum;            // [n_qt] (min anchor, max anchor, min depth, max depth)
+    int4 *ksum;            // [n_kt]
+    uint8_t *cls;          // [n_qt][n_kt] tile classes
+    int *undecided;        // [n_qt*n_kt] pairs the quick test could not decide
+    int *counters;         // [8] device counters (0: undecided, 1: bwd items, 2: bwd work cursor, 3: fwd cursor)
+    int2 *klist;           // [n_qt][n_kt] compact non-skip key tiles per query tile: (first token, len | cls<<16)
+    int *kcount;           // [n_qt]
+    int *qorder;           // [n_qt] query tiles, most key tiles first
+    int2 *qlist;           // [n_kt][n_qt] compact non-skip query tiles per key tile: (qt, cls)
+    int *qcount;           // [n_kt]
+    int4 *bitems;          // [n_kt * ceil(n_qt/BWD_CQ)] backward work items (kt, first list entry, n entries, -)
+    int *status;           // device status word
+};
+
+struct FwdArgs {
+    const void *Q, *K, *V;
+    void *O;
+    float *LSE;
+    int Hq, Hkv, D;
+    float scale;
+};
+
+struct BwdArgs {
+    const void *Q, *K, *V, *O, *dO;
+    const float *LSE;
+    void *dQ;
+    float *dK_acc, *dV_acc;
+    float *delta;   // [Hq][q_len] scratch
+    float *dq_acc;  // [q_len][Hq][D] scratch, fp32
+    int Hq, Hkv, D;
+    float scale;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// K0: mask evaluator, tile classifier, scheduler.  Returns the number of kernels launched.
+int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int K, int seq_begin,
+                int seq_end, const RangeList &ranges, bool for_bwd, int Hkv, cudaStream_t s);
+int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s);
+
+// K1 / K2.  Return the number of kernels launched, or a negative peagle_status.
+int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s);
+int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s);
+int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
+                      cudaStream_t s);
+
+// Packed-metadata form of the attention predicate: m = anchor << 8 | depth.
+// (depth_k == 0 and anchor_k <= anchor_q) or (anchor_k == anchor_q and depth_k <= depth_q)
+__host__ __device__ inline bool allowed_packed(int32_t mq, int32_t mk)
+{
+    return (mk <= mq) && (((mk & 0xff) == 0) || ((mk ^ mq) < 256));
+}
+
+} // namespace peagle

@@ -1,0 +1,336 @@
+// K0: implicit mask evaluator, tile classifier and scheduler.
+//
+// The parallel-prediction mask (paper Section 3 / 3.2) is a function of per-token metadata only,
+// so it is evaluated from a packed word per token (anchor << 8 | depth) and never stored.  For
+// one call (a query partition and the key ranges it may see) these kernels
+//   1. pack and validate the metadata and lay out the key tiles of the visible ranges,
+//   2. summarise every query tile and key tile (min/max anchor and depth),
+//   3. classify every (query tile, key tile) pair as SKIP / PARTIAL / FULL -- from the summaries
+//      where they decide, else exactly by evaluating the predicate on the tile,
+//   4. compact the non-skipped tiles into per-query-tile lists (forward) and per-key-tile lists
+//      (backward), order query tiles longest-first and cut the backward into work items.
+// Everything runs on the caller's stream; nothing returns to the host.
+#include "peagle_internal.h"
+
+namespace peagle {
+
+__device__ __forceinline__ void set_status(int *status, int err)
+{
+    atomicCAS(status, 0, err);
+}
+
+// ---- 1. pack metadata, build key tiles ---------------------------------------------------
+__global__ void k0_prepare(Plan p, const int32_t *__restrict__ anchor,
+                           const int32_t *__restrict__ depth, int K, int seq_begin, int seq_end,
+                           RangeList ranges)
+{
+    const int t = seq_begin + blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < seq_end) {
+        const int a = anchor[t], d = depth[t];
+        if (a < 0 || a >= (1 << 23) || d < 0 || d >= K) {
+            set_status(p.status, PEAGLE_ERR_BAD_META);
+            p.meta[t] = META_NONE_K;
+        } else {
+            p.meta[t] = (a << 8) | d;
+        }
+    }
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        int kt = 0;
+        for (int i = 0; i < ranges.n; ++i)
+            for (int b = ranges.begin[i]; b < ranges.end[i]; b += BN, ++kt)
+                p.ktile[kt] = make_int2(b, min(BN, ranges.end[i] - b));
+        for (int i = 0; i < 8; ++i)
+            p.counters[i] = 0;
+    }
+}
+
+// ---- 2. tile summaries -----------------------------------------------------------------
+__global__ void k0_summaries(Plan p)
+{
+    const int tile = blockIdx.x;
+    int b, e;
+    int4 *out;
+    if (tile < p.n_qt) {
+        b = p.q_begin + tile * BM;
+        e = min(b + BM, p.q_end);
+        out = p.qsum + tile;
+    } else {
+        const int2 kt = p.ktile[tile - p.n_qt];
+        b = kt.x;
+        e = kt.x + kt.y;
+        out = p.ksum + (tile - p.n_qt);
+    }
+    int a0 = INT_MAX, a1 = -1, d0 = INT_MAX, d1 = -1;
+    const int t = b + threadIdx.x;
+    if (t < e) {
+        const int m = p.meta[t];
+        if (m != META_NONE_K) {
+            a0 = a1 = m >> 8;
+            d0 = d1 = m & 0xff;
+        }
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        a0 = min(a0, __shfl_xor_sync(0xffffffffu, a0, o));
+        a1 = max(a1, __shfl_xor_sync(0xffffffffu, a1, o));
+        d0 = min(d0, __shfl_xor_sync(0xffffffffu, d0, o));
+        d1 = max(d1, __shfl_xor_sync(0xffffffffu, d1, o));
+    }
+    __shared__ int4 part[4];
+    if ((threadIdx.x & 31) == 0)
+        part[threadIdx.x >> 5] = make_int4(a0, a1, d0, d1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int4 r = part[0];
+        for (int w = 1; w < 4; ++w) {
+            r.x = min(r.x, part[w].x);
+            r.y = max(r.y, part[w].y);
+            r.z = min(r.z, part[w].z);
+            r.w = max(r.w, part[w].w);
+        }
+        *out = r;
+    }
+}
+
+// ---- 3a. classification from summaries ---------------------------------------------------
+__global__ void k0_classify_quick(Plan p)
+{
+    const int kt = blockIdx.x * blockDim.x + threadIdx.x;
+    const int qt = blockIdx.y;
+    if (kt >= p.n_kt)
+        return;
+    const int4 q = p.qsum[qt];
+    const int4 k = p.ksum[kt];
+    const int len = p.ktile[kt].y;
+    int c = -1;
+    if (k.y < 0 || q.y < 0) {
+        c = TILE_SKIP; // a tile with no valid token
+    } else if (k.w == 0) { // every key is a depth-0 (real context) token
+        if (k.y <= q.x)
+            c = (len == BN) ? TILE_FULL : TILE_PARTIAL;
+        else if (k.x > q.y)
+            c = TILE_SKIP;
+    } else if (k.z >= 1) { // no depth-0 key: only same-anchor, not-deeper chain tokens can match
+        if (k.x > q.y || k.y < q.x || k.z > q.w)
+            c = TILE_SKIP;
+    }
+    const size_t idx = (size_t)qt * p.n_kt + kt;
+    if (c >= 0) {
+        p.cls[idx] = (uint8_t)c;
+    } else {
+        p.cls[idx] = 255;
+        p.undecided[atomicAdd(&p.counters[0], 1)] = (int)idx;
+    }
+}
+
+// ---- 3b. exact classification of the remaining pairs ------------------------------------
+__global__ void k0_classify_exact(Plan p)
+{
+    __shared__ int mk[BN];
+    __shared__ int total;
+    const int n = p.counters[0];
+    for (int w = blockIdx.x; w < n; w += gridDim.x) {
+        const int idx = p.undecided[w];
+        const int qt = idx / p.n_kt, kt = idx % p.n_kt;
+        const int2 ktile = p.ktile[kt];
+        const int r0 = p.q_begin + qt * BM, r1 = min(r0 + BM, p.q_end);
+        __syncthreads();
+        mk[threadIdx.x] = ((int)threadIdx.x < ktile.y) ? p.meta[ktile.x + threadIdx.x] : META_NONE_K;
+        if (threadIdx.x == 0)
+            total = 0;
+        __syncthreads();
+        int cnt = 0;
+        if (r0 + (int)threadIdx.x < r1) {
+            const int mq = p.meta[r0 + threadIdx.x];
+            if (mq != META_NONE_K)
+                for (int c = 0; c < BN; ++c)
+                    cnt += allowed_packed(mq, mk[c]);
+        }
+        for (int o = 16; o > 0; o >>= 1)
+            cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
+        if ((threadIdx.x & 31) == 0)
+            atomicAdd(&total, cnt);
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint8_t c = TILE_PARTIAL;
+            if (total == 0)
+                c = TILE_SKIP;
+            else if (ktile.y == BN && total == (r1 - r0) * BN)
+                c = TILE_FULL;
+            p.cls[idx] = c;
+        }
+    }
+}
+
+// ---- 4a. compact lists -------------------------------------------------------------------
+// Blocks [0, n_qt): key-tile list of a query tile.  Blocks [n_qt, n_qt + n_kt): query-tile list
+// of a key tile (backward only).  Order inside a list is ascending tile index.
+__global__ void k0_lists(Plan p, int for_bwd)
+{
+    __shared__ int warp_cnt[4];
+    __shared__ int base;
+    const bool is_q = (int)blockIdx.x < p.n_qt;
+    if (!is_q && !for_bwd)
+        return;
+    const int self = is_q ? blockIdx.x : blockIdx.x - p.n_qt;
+    const int n_other = is_q ? p.n_kt : p.n_qt;
+    if (threadIdx.x == 0)
+        base = 0;
+    __syncthreads();
+    for (int o0 = 0; o0 < n_other; o0 += blockDim.x) {
+        const int o = o0 + threadIdx.x;
+        uint8_t c = TILE_SKIP;
+        if (o < n_other)
+            c = is_q ? p.cls[(size_t)self * p.n_kt + o] : p.cls[(size_t)o * p.n_kt + self];
+        const unsigned bal = __ballot_sync(0xffffffffu, c != TILE_SKIP);
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+        if (lane == 0)
+            warp_cnt[wid] = __popc(bal);
+        __syncthreads();
+        int off = base;
+        for (int w = 0; w < wid; ++w)
+            off += warp_cnt[w];
+        off += __popc(bal & ((1u << lane) - 1u));
+        if (c != TILE_SKIP) {
+            if (is_q) {
+                const int2 kt = p.ktile[o];
+                p.klist[(size_t)self * p.n_kt + off] = make_int2(kt.x, kt.y | ((int)c << 16));
+            } else {
+                p.qlist[(size_t)self * p.n_qt + off] = make_int2(o, (int)c);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0)
+            base += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        if (is_q)
+            p.kcount[self] = base;
+        else
+            p.qcount[self] = base;
+    }
+}
+
+// ---- 4b. order query tiles longest-first; cut the backward into work items ------------------
+__global__ void k0_schedule(Plan p, int for_bwd)
+{
+    extern __shared__ int cnt[];
+    const int n = p.n_qt;
+    if (n <= 8192) {
+        for (int i = threadIdx.x; i < n; i += blockDim.x)
+            cnt[i] = p.kcount[i];
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int ci = cnt[i];
+            int rank = 0;
+            for (int j = 0; j < n; ++j)
+                rank += (cnt[j] > ci) || (cnt[j] == ci && j < i);
+            p.qorder[rank] = i;
+        }
+    } else {
+        for (int i = threadIdx.x; i < n; i += blockDim.x)
+            p.qorder[i] = n - 1 - i;
+    }
+    if (!for_bwd)
+        return;
+    // Work item = one key tile and up to BWD_CQ consecutive entries of its query-tile list.
+    // Key tiles with long lists come first because their items are all full-sized.
+    __shared__ int sum_big[1024], sum_small[1024];
+    __shared__ int total_big;
+    const int per = (p.n_kt + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int k0 = min(p.n_kt, (int)threadIdx.x * per), k1 = min(p.n_kt, k0 + per);
+    int nb = 0, ns = 0;
+    for (int kt = k0; kt < k1; ++kt) {
+        const int c = p.qcount[kt];
+        const int chunks = (c + BWD_CQ - 1) / BWD_CQ;
+        if (c >= BWD_CQ)
+            nb += chunks;
+        else
+            ns += chunks;
+    }
+    sum_big[threadIdx.x] = nb;
+    sum_small[threadIdx.x] = ns;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int ab = 0, as = 0;
+        for (int i = 0; i < (int)blockDim.x; ++i) {
+            const int b = sum_big[i], sm = sum_small[i];
+            sum_big[i] = ab;
+            sum_small[i] = as;
+            ab += b;
+            as += sm;
+        }
+        total_big = ab;
+        p.counters[1] = ab + as;
+    }
+    __syncthreads();
+    int ob = sum_big[threadIdx.x], os = total_big + sum_small[threadIdx.x];
+    for (int kt = k0; kt < k1; ++kt) {
+        const int c = p.qcount[kt];
+        for (int j = 0; j < c; j += BWD_CQ) {
+            const int4 item = make_int4(kt, j, min(BWD_CQ, c - j), 0);
+            if (c >= BWD_CQ)
+                p.bitems[ob++] = item;
+            else
+                p.bitems[os++] = item;
+        }
+    }
+}
+
+// ---- test hook: the mask as the device predicate sees it -----------------------------------
+__global__ void k0_mask_dense(Plan p, RangeList ranges, uint8_t *out)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    const int q = p.q_begin + blockIdx.y;
+    if (k >= p.T)
+        return;
+    bool vis = false;
+    for (int i = 0; i < ranges.n; ++i)
+        vis |= (k >= ranges.begin[i] && k < ranges.end[i]);
+    const int mq = p.meta[q], mk = p.meta[k];
+    out[(size_t)blockIdx.y * p.T + k] =
+        (uint8_t)(vis && mq != META_NONE_K && allowed_packed(mq, mk));
+}
+
+// No visible key: every query tile has an empty list.
+__global__ void k0_empty(Plan p)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < p.n_qt) {
+        p.kcount[i] = 0;
+        p.qorder[i] = i;
+    }
+}
+
+int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int K, int seq_begin,
+                int seq_end, const RangeList &ranges, bool for_bwd, int Hkv, cudaStream_t s)
+{
+    (void)Hkv;
+    const int n_seq = seq_end - seq_begin;
+    k0_prepare<<<(n_seq + 255) / 256 > 0 ? (n_seq + 255) / 256 : 1, 256, 0, s>>>(
+        p, anchor, depth, K, seq_begin, seq_end, ranges);
+    if (p.n_qt == 0)
+        return 1;
+    if (p.n_kt == 0) {
+        k0_empty<<<(p.n_qt + 255) / 256, 256, 0, s>>>(p);
+        return 2;
+    }
+    k0_summaries<<<p.n_qt + p.n_kt, 128, 0, s>>>(p);
+    k0_classify_quick<<<dim3((p.n_kt + 127) / 128, p.n_qt), 128, 0, s>>>(p);
+    k0_classify_exact<<<592, 128, 0, s>>>(p);
+    k0_lists<<<p.n_qt + (for_bwd ? p.n_kt : 0), 128, 0, s>>>(p, for_bwd ? 1 : 0);
+    const int smem = (p.n_qt <= 8192 ? p.n_qt : 0) * (int)sizeof(int);
+    k0_schedule<<<1, 1024, smem, s>>>(p, for_bwd ? 1 : 0);
+    return 6;
+}
+
+int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s)
+{
+    const int q_len = p.q_end - p.q_begin;
+    if (q_len <= 0)
+        return 0;
+    k0_mask_dense<<<dim3((p.T + 255) / 256, q_len), 256, 0, s>>>(p, ranges, out);
+    return 1;
+}
+
+} // namespace peagle

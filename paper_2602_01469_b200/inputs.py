@@ -127,3 +127,36 @@ def make_tensors(T: int, Hq: int, Hkv: int, D: int, seed: int, q_std: float | No
         g.manual_seed(seed * 10 + i + 1)
         out.append((torch.randn(T, H, D, generator=g, dtype=torch.float32) * s).to(torch.bfloat16))
     return tuple(out)  # Q, K, V, dO
+
+
+def build_case(w: Workload, assign_fn):
+    """Lays out a workload: per sequence the full grid of anchors x depths, segments from
+    ``assign_fn(anchor, depth, K, boundaries) -> segment per token`` (Algorithm 1, supplied by the
+    caller: the library's or the oracle's), tokens ordered by (segment, depth, anchor).
+    Returns cu_seqlens, anchor, depth (int32 arrays in memory order) and the partitions as
+    dicts {seq, q: (b, e), k: [(b, e), ...]} in execution order."""
+    cu = [0]
+    anchors, depths, parts = [], [], []
+    for i, n in enumerate(w.seq_lens):
+        a, d = full_grid(n, w.K)
+        bounds = segment_boundaries(n, w.n_segments, w.seg_len)
+        if len(bounds) > 2:
+            seg = np.asarray(assign_fn(a, d, w.K, bounds), dtype=np.int32)
+        else:
+            seg = np.zeros(a.shape[0], np.int32)
+        perm = arrange_by_segment(a, d, seg)
+        a, d, seg = a[perm], d[perm], seg[perm]
+        for p in partitions_from_layout(seg, d, offset=cu[-1]):
+            p["seq"] = i
+            parts.append(p)
+        anchors.append(a)
+        depths.append(d)
+        cu.append(cu[-1] + a.shape[0])
+    return (np.asarray(cu, np.int32), np.concatenate(anchors).astype(np.int32),
+            np.concatenate(depths).astype(np.int32), parts)
+
+
+def allowed_pairs_full_grid(n: int, K: int) -> int:
+    """Number of (query, key) pairs the mask allows on a full grid: a token at position
+    anchor+depth sees anchor+1 real tokens and `depth` chain tokens."""
+    return K * n * (n + 1) // 2 + n * K * (K - 1) // 2
