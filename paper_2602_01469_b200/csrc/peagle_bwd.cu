@@ -1,6 +1,577 @@
-// K2 placeholder
+// K2: backward of one query partition on sm_100a (dQ, and fp32 accumulation of dK / dV).
+//
+// Key-tile-outer formulation.  A work item is one key tile (128 keys) of one KV head together
+// with up to BWD_CQ query tiles of its list; for each of those query tiles the item visits the
+// G query heads of the group.  dK and dV of the key tile stay in tensor memory for the whole item
+// and are added to the caller's fp32 accumulators once at its end; dQ of each visited (query
+// tile, head) is added to an fp32 staging buffer and rounded to bf16 by a last kernel.
+//
+// All score-shaped matrices are held transposed (lanes = keys, columns = query rows) so that the
+// probabilities can feed the dV product straight from tensor memory:
+//   S^T  = K Q^T            both operands from shared memory (K-major)
+//   dP^T = V dO^T           both operands from shared memory (K-major)
+//   P^T  = exp2(scale*log2e*S^T - LSE*log2e), masked entries 0;  dS^T = P^T o (dP^T - Delta)
+//   dV  += P^T dO           P^T from tensor memory (bf16, over S^T), dO from shared memory (MN-major)
+//   dK  += dS^T Q           dS^T from shared memory (K-major), Q MN-major
+//   dQ   = dS K             dS^T read as an MN-major A operand, K MN-major
+// Roles: warps 0-7 compute (two groups of 128 threads, one key per thread, each group half of
+// the query columns), warp 8 lane 0 issues the MMAs, warp 9 is the TMA producer.
+#include <math_constants.h>
+
 #include "peagle_internal.h"
+#include "sm100_ptx.cuh"
+
 namespace peagle {
-int launch_bwd(const Plan &, const BwdArgs &, EncodeTiledFn, int, cudaStream_t) { return 0; }
-int launch_cast_grads(const float *, const float *, void *, void *, size_t, cudaStream_t) { return 0; }
+using namespace sm100;
+
+int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int H, int T);
+
+struct BwdParams {
+    const int2 *ktile;
+    const int2 *qlist;
+    const int4 *bitems;
+    const int *counters;
+    const int32_t *meta;
+    int *status;
+    int n_qt, q_begin, q_end, T;
+    const float *LSE;
+    const float *delta; // [Hq][q_len]
+    float *dq_acc;      // [q_len][Hq][D]
+    float *dK_acc, *dV_acc;
+    int Hq, Hkv;
+    float scale, scale_log2;
+};
+
+template <int D>
+struct BwdCfg {
+    static constexpr int NSQ = (D == 64) ? 2 : 1;
+    static constexpr int PANELS = D / 64;
+    static constexpr int PANEL_BYTES = 128 * 128;
+    static constexpr int TILE_BYTES = PANELS * PANEL_BYTES;
+    static constexpr int OFF_K = 0;
+    static constexpr int OFF_V = TILE_BYTES;
+    static constexpr int OFF_DS = 2 * TILE_BYTES;                 // 2 panels: [key][q 0..63], [key][q 64..127]
+    static constexpr int OFF_Q = OFF_DS + 2 * PANEL_BYTES;        // ring of (Q, dO)
+    static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (lse2[128], delta[128], mq[128])
+    static constexpr int ROW_BYTES = 3 * 128 * 4;
+    static constexpr int OFF_BAR = OFF_ROW + NSQ * ROW_BYTES;
+    static constexpr int N_BAR = 2 * NSQ + 9;
+    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
+    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
+    static constexpr int TM_S = 0;
+    static constexpr int TM_DP = 128;
+    static constexpr int TM_DQ = (D == 64) ? 256 : 128; // head_dim 128: dQ reuses the dP columns
+    static constexpr int TM_DK = (D == 64) ? 320 : 256;
+    static constexpr int TM_DV = (D == 64) ? 384 : 384;
+};
+
+__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c),
+                 "f"(d)
+                 : "memory");
 }
+
+template <int D>
+__global__ void __launch_bounds__(320, 1)
+bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
+           const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+           const BwdParams P)
+{
+    using C = BwdCfg<D>;
+    constexpr int NSQ = C::NSQ;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u;
+    uint8_t *sp = smem_raw + (sb - raw);
+    const uint32_t bar0 = sb + C::OFF_BAR;
+    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    constexpr int B_QFULL = 0, B_QEMPTY = NSQ, B_KVFULL = 2 * NSQ, B_KVEMPTY = B_KVFULL + 1,
+                  B_ACCFREE = B_KVFULL + 2, B_SFULL = B_KVFULL + 3, B_DPFULL = B_KVFULL + 4,
+                  B_PFULL = B_KVFULL + 5, B_DSFULL = B_KVFULL + 6, B_DQFULL = B_KVFULL + 7,
+                  B_DQEMPTY = B_KVFULL + 8;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int G = P.Hq / P.Hkv;
+    const int total_items = P.counters[1] * P.Hkv;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < NSQ; ++s) {
+            mbar_init(BAR(B_QFULL + s), 1);
+            mbar_init(BAR(B_QEMPTY + s), 1);
+        }
+        mbar_init(BAR(B_KVFULL), 1);
+        mbar_init(BAR(B_KVEMPTY), 1);
+        mbar_init(BAR(B_ACCFREE), 256);
+        mbar_init(BAR(B_SFULL), 1);
+        mbar_init(BAR(B_DPFULL), 1);
+        mbar_init(BAR(B_PFULL), 256);
+        mbar_init(BAR(B_DSFULL), 256);
+        mbar_init(BAR(B_DQFULL), 1);
+        mbar_init(BAR(B_DQEMPTY), 256);
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(sb + C::OFF_MISC, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 9) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmQ);
+            tma_prefetch_desc(&tmdO);
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+        }
+        int it = 0, w = 0;
+        bool ok = true;
+        for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
+            const int4 item = P.bitems[idx / P.Hkv];
+            const int g = idx % P.Hkv;
+            const int kt = item.x;
+            const int2 ktile = P.ktile[kt];
+            if (lane == 0) {
+                ok = mbar_wait(BAR(B_KVEMPTY), (w & 1) ^ 1, abort_flag);
+                if (ok) {
+                    mbar_arrive_expect_tx(BAR(B_KVFULL), 2 * C::TILE_BYTES);
+                    for (int pn = 0; pn < C::PANELS; ++pn) {
+                        tma_load_3d(sb + C::OFF_K + pn * C::PANEL_BYTES, &tmK, BAR(B_KVFULL), pn * 64,
+                                    g, ktile.x);
+                        tma_load_3d(sb + C::OFF_V + pn * C::PANEL_BYTES, &tmV, BAR(B_KVFULL), pn * 64,
+                                    g, ktile.x);
+                    }
+                }
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            for (int e = 0; ok && e < item.z; ++e) {
+                const int qt = P.qlist[(size_t)kt * P.n_qt + item.y + e].x;
+                const int row0 = P.q_begin + qt * BM;
+                for (int hh = 0; ok && hh < G; ++hh, ++it) {
+                    const int h = g * G + hh;
+                    const int st = it % NSQ, ph = (it / NSQ) & 1;
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
+                    if (!ok)
+                        break;
+                    float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
+                    for (int i = lane; i < BM; i += 32) {
+                        const int row = row0 + i;
+                        float l2 = CUDART_INF_F, dl = 0.f;
+                        int mq = META_NONE_Q;
+                        if (row < P.q_end) {
+                            const float lse = P.LSE[(size_t)h * P.T + row];
+                            if (lse != -CUDART_INF_F)
+                                l2 = lse * 1.4426950408889634f;
+                            dl = P.delta[(size_t)h * (P.q_end - P.q_begin) + (row - P.q_begin)];
+                            mq = P.meta[row];
+                            if (mq == META_NONE_K)
+                                mq = META_NONE_Q;
+                        }
+                        rowbuf[i] = l2;
+                        rowbuf[128 + i] = dl;
+                        reinterpret_cast<int *>(rowbuf)[256 + i] = mq;
+                    }
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * C::TILE_BYTES);
+                        const uint32_t qa = sb + C::OFF_Q + st * 2 * C::TILE_BYTES;
+                        for (int pn = 0; pn < C::PANELS; ++pn) {
+                            tma_load_3d(qa + pn * C::PANEL_BYTES, &tmQ, BAR(B_QFULL + st), pn * 64, h,
+                                        row0);
+                            tma_load_3d(qa + C::TILE_BYTES + pn * C::PANEL_BYTES, &tmdO,
+                                        BAR(B_QFULL + st), pn * 64, h, row0);
+                        }
+                    }
+                }
+            }
+        }
+    } else if (warp == 8) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
+            constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
+            constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
+            const uint32_t ka = sb + C::OFF_K, va = sb + C::OFF_V, dsa = sb + C::OFF_DS;
+            int it = 0, w = 0;
+            bool ok = true;
+            for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
+                const int4 item = P.bitems[idx / P.Hkv];
+                const int n_it = item.z * G;
+                ok = mbar_wait(BAR(B_KVFULL), w & 1, abort_flag) &&
+                     mbar_wait(BAR(B_ACCFREE), (w & 1) ^ 1, abort_flag);
+                for (int i = 0; ok && i < n_it; ++i, ++it) {
+                    const int st = it % NSQ, ph = (it / NSQ) & 1;
+                    const uint32_t qa = sb + C::OFF_Q + st * 2 * C::TILE_BYTES;
+                    const uint32_t doa = qa + C::TILE_BYTES;
+                    ok = mbar_wait(BAR(B_QFULL + st), ph, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
+                        mma_ss(tmem + C::TM_S, smem_desc_sw128(ka + off, 16, 1024),
+                               smem_desc_sw128(qa + off, 16, 1024), IDESC_S, k > 0);
+                    }
+                    tc_commit(BAR(B_SFULL));
+                    if (D == 128) { // dQ of the previous iteration lives in the dP columns
+                        ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, abort_flag);
+                        if (!ok)
+                            break;
+                        tc_fence_after();
+                    }
+#pragma unroll
+                    for (int k = 0; k < D / 16; ++k) {
+                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
+                        mma_ss(tmem + C::TM_DP, smem_desc_sw128(va + off, 16, 1024),
+                               smem_desc_sw128(doa + off, 16, 1024), IDESC_S, k > 0);
+                    }
+                    tc_commit(BAR(B_DPFULL));
+                    ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mma_ts(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                               smem_desc_sw128(doa + k * 2048, C::PANEL_BYTES, 1024), IDESC_KV,
+                               i > 0 || k > 0);
+                    ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag);
+                    if (ok && D == 64)
+                        ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
+                        mma_ss(tmem + C::TM_DK, smem_desc_sw128(dsa + off, 16, 1024),
+                               smem_desc_sw128(qa + k * 2048, C::PANEL_BYTES, 1024), IDESC_KV,
+                               i > 0 || k > 0);
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss(tmem + C::TM_DQ, smem_desc_sw128(dsa + k * 2048, C::PANEL_BYTES, 1024),
+                               smem_desc_sw128(ka + k * 2048, C::PANEL_BYTES, 1024), IDESC_DQ, k > 0);
+                    tc_commit(BAR(B_DQFULL));
+                    tc_commit(BAR(B_QEMPTY + st));
+                }
+                if (ok)
+                    tc_commit(BAR(B_KVEMPTY));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ compute (warps 0-7)
+        const int wg = warp >> 2;
+        const int r = threadIdx.x & 127; // key lane for S/dP/dK/dV, query row for dQ
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_sel + C::TM_S + wg * 64;
+        const uint32_t tDP = tmem + lane_sel + C::TM_DP + wg * 64;
+        const uint32_t tDQ = tmem + lane_sel + C::TM_DQ + wg * (D / 2);
+        const uint32_t tACC = tmem + lane_sel + (wg == 0 ? C::TM_DK : C::TM_DV);
+        const size_t q_len = (size_t)(P.q_end - P.q_begin);
+        int it = 0, w = 0;
+        bool ok = true;
+        for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
+            const int4 item = P.bitems[idx / P.Hkv];
+            const int g = idx % P.Hkv;
+            const int kt = item.x;
+            const int2 ktile = P.ktile[kt];
+            const int32_t mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
+            for (int e = 0; ok && e < item.z; ++e) {
+                const int2 qe = P.qlist[(size_t)kt * P.n_qt + item.y + e];
+                const int row0 = P.q_begin + qe.x * BM;
+                const bool full = qe.y == TILE_FULL;
+                for (int hh = 0; ok && hh < G; ++hh, ++it) {
+                    const int h = g * G + hh;
+                    const int st = it % NSQ, ph = (it / NSQ) & 1;
+                    const float *rowbuf =
+                        reinterpret_cast<const float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
+                    const float4 *lse4 = reinterpret_cast<const float4 *>(rowbuf + wg * 64);
+                    const float4 *dl4 = reinterpret_cast<const float4 *>(rowbuf + 128 + wg * 64);
+                    const int4 *mq4 = reinterpret_cast<const int4 *>(rowbuf + 256 + wg * 64);
+                    // ---- P^T
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL), it & 1, abort_flag) &&
+                                                     mbar_wait(BAR(B_QFULL + st), ph, abort_flag));
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    uint32_t sr[2][32];
+                    tmem_ld32(tS, sr[0]);
+                    tmem_ld32(tS + 32, sr[1]);
+                    tmem_wait_ld();
+                    float p[64];
+#pragma unroll
+                    for (int c = 0; c < 64; c += 4) {
+                        const float4 l = lse4[c >> 2];
+                        p[c + 0] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 0) & 31]), P.scale_log2, -l.x));
+                        p[c + 1] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 1) & 31]), P.scale_log2, -l.y));
+                        p[c + 2] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 2) & 31]), P.scale_log2, -l.z));
+                        p[c + 3] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 3) & 31]), P.scale_log2, -l.w));
+                    }
+                    if (!full) {
+#pragma unroll
+                        for (int c = 0; c < 64; c += 4) {
+                            const int4 mq = mq4[c >> 2];
+                            if (!allowed_packed(mq.x, mk)) p[c + 0] = 0.f;
+                            if (!allowed_packed(mq.y, mk)) p[c + 1] = 0.f;
+                            if (!allowed_packed(mq.z, mk)) p[c + 2] = 0.f;
+                            if (!allowed_packed(mq.w, mk)) p[c + 3] = 0.f;
+                        }
+                    }
+                    {
+                        uint32_t pk[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            pk[i] = pack_bf16x2(p[2 * i], p[2 * i + 1]);
+                        tmem_st32(tS, pk); // packed P^T over the first half of this group's S^T columns
+                    }
+                    tmem_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(BAR(B_PFULL));
+                    // ---- dS^T
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DPFULL), it & 1, abort_flag));
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    tmem_ld32(tDP, sr[0]);
+                    tmem_ld32(tDP + 32, sr[1]);
+                    tmem_wait_ld();
+                    {
+                        uint8_t *dsrow = sp + C::OFF_DS + wg * C::PANEL_BYTES + r * 128;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { // 16-byte chunk j = query columns 8j .. 8j+7
+                            const float4 d0 = dl4[2 * j], d1 = dl4[2 * j + 1];
+                            const int c = 8 * j;
+                            uint4 v;
+                            v.x = pack_bf16x2(p[c + 0] * (__uint_as_float(sr[c >> 5][(c + 0) & 31]) - d0.x),
+                                              p[c + 1] * (__uint_as_float(sr[c >> 5][(c + 1) & 31]) - d0.y));
+                            v.y = pack_bf16x2(p[c + 2] * (__uint_as_float(sr[c >> 5][(c + 2) & 31]) - d0.z),
+                                              p[c + 3] * (__uint_as_float(sr[c >> 5][(c + 3) & 31]) - d0.w));
+                            v.z = pack_bf16x2(p[c + 4] * (__uint_as_float(sr[c >> 5][(c + 4) & 31]) - d1.x),
+                                              p[c + 5] * (__uint_as_float(sr[c >> 5][(c + 5) & 31]) - d1.y));
+                            v.w = pack_bf16x2(p[c + 6] * (__uint_as_float(sr[c >> 5][(c + 6) & 31]) - d1.z),
+                                              p[c + 7] * (__uint_as_float(sr[c >> 5][(c + 7) & 31]) - d1.w));
+                            *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = v;
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    tc_fence_before();
+                    mbar_arrive(BAR(B_DSFULL));
+                    // ---- dQ of this (query tile, head): add to the fp32 staging buffer
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DQFULL), it & 1, abort_flag));
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    {
+                        const int row = row0 + r;
+                        float *dst = P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D + wg * (D / 2);
+#pragma unroll
+                        for (int c = 0; c < D / 64; ++c) {
+                            uint32_t o[32];
+                            tmem_ld32(tDQ + c * 32, o);
+                            tmem_wait_ld();
+                            if (row < P.q_end) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 4)
+                                    red_add_v4(dst + c * 32 + i, __uint_as_float(o[i]) * P.scale,
+                                               __uint_as_float(o[i + 1]) * P.scale,
+                                               __uint_as_float(o[i + 2]) * P.scale,
+                                               __uint_as_float(o[i + 3]) * P.scale);
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    mbar_arrive(BAR(B_DQEMPTY));
+                }
+            }
+            if (!ok)
+                break;
+            // ---- end of item: dK (group 0) / dV (group 1) of this key tile
+            {
+                float *acc = (wg == 0 ? P.dK_acc : P.dV_acc) +
+                             ((size_t)(ktile.x + r) * P.Hkv + g) * D;
+                const float f = (wg == 0) ? P.scale : 1.f;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tACC + c * 32, o);
+                    tmem_wait_ld();
+                    if (r < ktile.y) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            red_add_v4(acc + c * 32 + i, __uint_as_float(o[i]) * f,
+                                       __uint_as_float(o[i + 1]) * f, __uint_as_float(o[i + 2]) * f,
+                                       __uint_as_float(o[i + 3]) * f);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(BAR(B_ACCFREE));
+        }
+        (void)q_len;
+    }
+
+    // ------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {
+        }
+        __syncthreads();
+    }
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
+// Delta[h][r] = <dO[q,h,:], O[q,h,:]> for the rows of the partition, and zero the fp32 dQ staging.
+template <int D>
+__global__ void bwd_prepare(const __nv_bfloat16 *__restrict__ O, const __nv_bfloat16 *__restrict__ dO,
+                            float *__restrict__ delta, float *__restrict__ dq_acc, int q_begin,
+                            int q_len, int Hq)
+{
+    constexpr int TPR = D / 8; // threads per (row, head)
+    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t n = (size_t)q_len * Hq * TPR;
+    float acc = 0.f;
+    if (gid < n) {
+        const size_t src = (size_t)q_begin * Hq * D + gid * 8;
+        const uint4 a = *reinterpret_cast<const uint4 *>(O + src);
+        const uint4 b = *reinterpret_cast<const uint4 *>(dO + src);
+        const __nv_bfloat162 *pa = reinterpret_cast<const __nv_bfloat162 *>(&a);
+        const __nv_bfloat162 *pb = reinterpret_cast<const __nv_bfloat162 *>(&b);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 x = __bfloat1622float2(pa[i]), y = __bfloat1622float2(pb[i]);
+            acc += x.x * y.x + x.y * y.y;
+        }
+        float4 *z = reinterpret_cast<float4 *>(dq_acc + gid * 8);
+        z[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+        z[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int o = TPR / 2; o > 0; o >>= 1)
+        acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (gid < n && (gid % TPR) == 0) {
+        const size_t rh = gid / TPR;
+        const size_t r = rh / Hq, h = rh % Hq;
+        delta[h * (size_t)q_len + r] = acc;
+    }
+}
+
+__global__ void bwd_finish_dq(const float *__restrict__ dq_acc, __nv_bfloat16 *__restrict__ dQ,
+                              size_t n8)
+{
+    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= n8)
+        return;
+    const float4 a = reinterpret_cast<const float4 *>(dq_acc)[2 * gid];
+    const float4 b = reinterpret_cast<const float4 *>(dq_acc)[2 * gid + 1];
+    uint4 v;
+    v.x = pack_bf16x2(a.x, a.y);
+    v.y = pack_bf16x2(a.z, a.w);
+    v.z = pack_bf16x2(b.x, b.y);
+    v.w = pack_bf16x2(b.z, b.w);
+    reinterpret_cast<uint4 *>(dQ)[gid] = v;
+}
+
+__global__ void cast_grads_kernel(const float *__restrict__ a, const float *__restrict__ b,
+                                  __nv_bfloat16 *__restrict__ oa, __nv_bfloat16 *__restrict__ ob,
+                                  size_t n8)
+{
+    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gid >= 2 * n8)
+        return;
+    const float *src = gid < n8 ? a : b;
+    __nv_bfloat16 *dst = gid < n8 ? oa : ob;
+    const size_t i = gid < n8 ? gid : gid - n8;
+    const float4 x = reinterpret_cast<const float4 *>(src)[2 * i];
+    const float4 y = reinterpret_cast<const float4 *>(src)[2 * i + 1];
+    uint4 v;
+    v.x = pack_bf16x2(x.x, x.y);
+    v.y = pack_bf16x2(x.z, x.w);
+    v.z = pack_bf16x2(y.x, y.y);
+    v.w = pack_bf16x2(y.z, y.w);
+    reinterpret_cast<uint4 *>(dst)[i] = v;
+}
+
+template <int D>
+static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+{
+    // Q and dO maps end at the partition's last row so that rows past it read as zeros.
+    CUtensorMap tmQ, tmdO, tmK, tmV;
+    if (make_bf16_map(enc, &tmQ, a.Q, D, a.Hq, p.q_end) || make_bf16_map(enc, &tmdO, a.dO, D, a.Hq, p.q_end) ||
+        make_bf16_map(enc, &tmK, a.K, D, a.Hkv, p.T) || make_bf16_map(enc, &tmV, a.V, D, a.Hkv, p.T))
+        return PEAGLE_ERR_CUDA;
+    const int q_len = p.q_end - p.q_begin;
+    const size_t n_prep = (size_t)q_len * a.Hq * (D / 8);
+    bwd_prepare<D><<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
+        static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.delta,
+        a.dq_acc, p.q_begin, q_len, a.Hq);
+    int launches = 1;
+    if (p.n_kt > 0) {
+        BwdParams P;
+        P.ktile = p.ktile;
+        P.qlist = p.qlist;
+        P.bitems = p.bitems;
+        P.counters = p.counters;
+        P.meta = p.meta;
+        P.status = p.status;
+        P.n_qt = p.n_qt;
+        P.q_begin = p.q_begin;
+        P.q_end = p.q_end;
+        P.T = p.T;
+        P.LSE = a.LSE;
+        P.delta = a.delta;
+        P.dq_acc = a.dq_acc;
+        P.dK_acc = a.dK_acc;
+        P.dV_acc = a.dV_acc;
+        P.Hq = a.Hq;
+        P.Hkv = a.Hkv;
+        P.scale = a.scale;
+        P.scale_log2 = a.scale * 1.4426950408889634f;
+        static bool attr_set = false;
+        if (!attr_set) {
+            if (cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     BwdCfg<D>::SMEM_BYTES) != cudaSuccess)
+                return PEAGLE_ERR_CUDA;
+            attr_set = true;
+        }
+        bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+        ++launches;
+    }
+    bwd_finish_dq<<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
+        a.dq_acc, static_cast<__nv_bfloat16 *>(a.dQ) + (size_t)p.q_begin * a.Hq * D, n_prep);
+    return launches + 1;
+}
+
+int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+{
+    if (p.n_qt == 0)
+        return 0;
+    return a.D == 64 ? launch_bwd_t<64>(p, a, enc, n_sm, s) : launch_bwd_t<128>(p, a, enc, n_sm, s);
+}
+
+int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
+                      cudaStream_t s)
+{
+    const size_t n8 = n / 8;
+    cast_grads_kernel<<<(unsigned)((2 * n8 + 255) / 256), 256, 0, s>>>(
+        dK_acc, dV_acc, static_cast<__nv_bfloat16 *>(dK), static_cast<__nv_bfloat16 *>(dV), n8);
+    return 1;
+}
+
+} // namespace peagle
