@@ -1,0 +1,314 @@
+#!/usr/bin/env python
+"""Benchmark of the masked parallel-drafting attention hot path (mask evaluator + tile
+classifier + forward + backward + partition driver) on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+A step is one call of ``peagle_attn_partitioned`` over the whole workload.  The metric is useful
+(unmasked) TFLOP/s: 14 * P * head_dim * n_q_heads per step, P = allowed (query, key) pairs.
+With N > 1 every rank runs an independent replica of the workload on its own GPU (the path has
+no exchange step); the value is the sum over ranks divided by the slowest rank's time.
+``--impl reference`` times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_01469_b200 import inputs  # noqa: E402
+
+METRIC = "masked-attn fwd+bwd useful TFLOP/s"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
+
+
+def allowed_pairs(w: inputs.Workload) -> int:
+    """Allowed (query, key) pairs of a full-grid workload: a token (anchor a, depth d) sees the
+    a+1 real tokens up to its anchor and its d chain tokens."""
+    return sum(w.K * n * (n + 1) // 2 + n * w.K * (w.K - 1) // 2 for n in w.seq_lens)
+
+
+def useful_flops(w: inputs.Workload):
+    p = allowed_pairs(w)
+    fwd = 4 * p * w.head_dim * w.n_q_heads
+    bwd = 10 * p * w.head_dim * w.n_q_heads
+    return fwd, bwd
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.samples = []
+        self.stop = threading.Event()
+        self.th = threading.Thread(target=self._run, daemon=True)
+
+    def _once(self):
+        try:
+            out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                  "-i", str(self.idx)], capture_output=True, text=True, timeout=10).stdout
+            f = [x.strip() for x in out.strip().split(",")]
+            if len(f) >= 6:
+                self.samples.append((float(f[0]), float(f[1]), f[2:6]))
+        except Exception:
+            pass
+
+    def _run(self):
+        while not self.stop.is_set():
+            self._once()
+            self.stop.wait(0.1)
+
+    def __enter__(self):
+        self.th.start()
+        return self
+
+    def __exit__(self, *a):
+        self.stop.set()
+        self.th.join(timeout=15)
+        if not self.samples:
+            self._once()
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({n for s in self.samples for n, v in zip(names, s[2]) if v.lower() == "active"})
+        return {"sm_mhz": float(np.median([s[0] for s in self.samples])),
+                "sm_max_mhz": self.samples[0][1], "reasons": reasons, "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ CPU oracle arm
+def oracle_sample(w: inputs.Workload, budget_s: float, seed: int = 0):
+    """Times the fp64 oracle (forward + backward) on random query rows of the workload's longest
+    sequence, all heads, until about ``budget_s`` seconds are spent.  Returns useful TFLOP/s."""
+    from oracle import partition as opart
+    from oracle import peagle_oracle as orc
+
+    n = max(w.seq_lens)
+    anchor, depth = inputs.full_grid(n, w.K)
+    T = n * w.K
+    Q, K, V, dO = inputs.make_tensors(T, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed)
+    Qf, Kf, Vf, dOf = (t.float().numpy() for t in (Q, K, V, dO))
+    rng = np.random.default_rng(seed)
+    rows_done, pairs_done, t_spent = 0, 0, 0.0
+    chunk = max(8, orc.num_threads())
+    while t_spent < budget_s:
+        rows = np.sort(rng.choice(T, size=chunk, replace=False)).astype(np.int32)
+        t0 = time.perf_counter()
+        orc.attn_fwd(anchor, depth, Qf, Kf, Vf, w.scale, rows=rows)
+        orc.attn_bwd(anchor, depth, Qf, Kf, Vf, dOf, w.scale, rows=rows)
+        t_spent += time.perf_counter() - t0
+        rows_done += len(rows)
+        pairs_done += int(np.sum(anchor[rows] + 1 + depth[rows]))
+        if t_spent < budget_s / 8:
+            chunk *= 2
+    flops = 14 * pairs_done * w.head_dim * w.n_q_heads
+    return {"value": flops / t_spent / 1e12, "unit": UNIT, "cores": orc.num_threads(),
+            "kind": "oracle",
+            "sample": f"{rows_done} random query rows x {w.n_q_heads} heads of {w.name} "
+                      f"(n={n}, K={w.K}), fwd+bwd, {t_spent:.1f} s"}, t_spent, flops
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(w, per_step / 4)
+    tot_t, tot_f, last = 0.0, 0, None
+    for i in range(args.steps):
+        last, t, f = oracle_sample(w, per_step, seed=i + 1)
+        tot_t += t
+        tot_f += f
+    value = tot_f / tot_t / 1e12
+    last["value"] = value
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "note": "each step is a bounded sample "
+                                        "of query rows; the value is useful FLOPs of the sample / time"},
+        "cpu_baseline": last,
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+# ------------------------------------------------------------------ CUDA arm
+def run_cuda(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2602_01469_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    ctx = binding.Context(local_rank)
+    cu, anchor, depth, parts = inputs.build_case(w, binding.peagle_assign_segments)
+    T = int(cu[-1])
+    Qc, Kc, Vc, dOc = inputs.make_tensors(T, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed)
+    Q, K, V, dO = (t.to(dev) for t in (Qc, Kc, Vc, dOc))
+    d_anchor, d_depth = torch.from_numpy(anchor).to(dev), torch.from_numpy(depth).to(dev)
+    O = torch.empty_like(Q)
+    dQ = torch.empty_like(Q)
+    dK, dV = torch.empty_like(K), torch.empty_like(V)
+    LSE = torch.empty(w.n_q_heads, T, dtype=torch.float32, device=dev)
+    prob = binding.Problem(cu, d_anchor, d_depth, w.K, w.n_q_heads, w.n_kv_heads, w.head_dim, w.scale)
+    bparts = [binding.Partition(p["seq"], p["q"], p["k"]) for p in parts]
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.peagle_attn_partitioned(ctx, prob, bparts, Q, K, V, dO, O, LSE, dQ, dK, dV, stream)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    if binding.peagle_poll_status(ctx) != 0:
+        raise RuntimeError("device-side error during warm-up")
+    binding.peagle_timing_enable(ctx, True)
+    binding.peagle_timing_read(ctx)
+    launches0 = binding.peagle_launch_count(ctx)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(local_rank) as clocks:
+        barrier()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        barrier()
+    ms_total = e0.elapsed_time(e1)
+    (k_fwd_ms, k_bwd_ms), (n_fwd, n_bwd) = binding.peagle_timing_read(ctx)
+    binding.peagle_timing_enable(ctx, False)
+    launches = binding.peagle_launch_count(ctx) - launches0
+    if binding.peagle_poll_status(ctx) != 0:
+        raise RuntimeError("device-side error during the timed region")
+    if world > 1:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    f_fwd, f_bwd = useful_flops(w)
+    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through the host entry point (pinned host buffers, copies timed)
+    hQ, hK, hV, hdO = (t.pin_memory() for t in (Qc, Kc, Vc, dOc))
+    hO, hdQ = torch.empty_like(hQ).pin_memory(), torch.empty_like(hQ).pin_memory()
+    hdK, hdV = torch.empty_like(hK).pin_memory(), torch.empty_like(hV).pin_memory()
+    hLSE = torch.empty(w.n_q_heads, T, dtype=torch.float32).pin_memory()
+    hprob = binding.Problem(cu, anchor, depth, w.K, w.n_q_heads, w.n_kv_heads, w.head_dim, w.scale)
+
+    def host_step():
+        binding.peagle_attn_partitioned_host(ctx, hprob, bparts, hQ, hK, hV, hdO, hO, hLSE, hdQ, hdK, hdV)
+
+    host_step()
+    barrier()
+    e2e_steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        host_step()
+    torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    nbytes = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))  # noqa: E731
+    h2d = nbytes(hQ, hK, hV, hdO) + 2 * anchor.nbytes
+    d2h = nbytes(hO, hLSE, hdQ, hdK, hdV)
+
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        peak = float(peaks["bf16_tflops"])
+        bwd_ms_launch = k_bwd_ms / max(n_bwd, 1)
+        fwd_ms_launch = k_fwd_ms / max(n_fwd, 1)
+        launches_per_step = max(n_bwd // args.steps, 1)
+        achieved = (f_bwd / launches_per_step) / (bwd_ms_launch * 1e-3) / 1e12
+        roofline = {
+            "kernel": "bwd_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
+            "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+            "peak_source": f"{peak_kind} bf16_tflops (burst)",
+            "ms_per_launch": bwd_ms_launch, "launches_timed": int(n_bwd),
+            "fwd_kernel": {"achieved": (f_fwd / launches_per_step) / (fwd_ms_launch * 1e-3) / 1e12,
+                           "ms_per_launch": fwd_ms_launch, "launches_timed": int(n_fwd)},
+            "step_frac_of_peak": value / world / peak,
+            "step_frac_of_sustained": value / world / float(peaks.get("bf16_tflops_sustained", peak)),
+        }
+        cpu, _, _ = oracle_sample(w, args.cpu_seconds) if world == 1 and args.cpu_seconds > 0 else (None, 0, 0)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "seq_lens": list(w.seq_lens) if len(w.seq_lens) < 4 else
+                       f"{len(w.seq_lens)} sequences", "K": w.K, "total_tokens": T,
+                       "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+                       "partitions": len(parts), "allowed_pairs": allowed_pairs(w),
+                       "useful_tflop_per_step": (f_fwd + f_bwd) / 1e12,
+                       "l2": "inputs (>1 GB) larger than L2, no flush", "parallelism": "replicas"},
+            "clocks": clocks.summary(),
+            "e2e": {"value": world * (f_fwd + f_bwd) / e2e_s / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s},
+            "gpu_launches": int(launches),
+            "roofline": roofline,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--workload", default=inputs.HEADLINE, choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--cpu-seconds", type=float, default=15.0,
+                    help="CPU time for the oracle baseline (0 = skip)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
+    w = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

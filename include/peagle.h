@@ -101,6 +101,16 @@ int peagle_tile_shape(const peagle_ctx *ctx, int head_dim, int *BM, int *BN);
 int peagle_poll_status(peagle_ctx *ctx, void *stream);
 /* Number of kernels this library has launched through `ctx` since creation. */
 int64_t peagle_launch_count(const peagle_ctx *ctx);
+/*
+ * Measurement hooks (no counterpart in the paper).  With timing on, every later call records a
+ * CUDA event pair on its stream around its forward kernel and around its backward kernel.
+ * peagle_timing_read synchronises the device, adds up the recorded intervals since the last
+ * read, writes ms_out[0] = forward-kernel milliseconds, ms_out[1] = backward-kernel
+ * milliseconds, n_out[0], n_out[1] = how many launches of each were timed, and forgets them.
+ * At most 4096 launches of each kind are kept between reads; later ones go untimed.
+ */
+int peagle_timing_enable(peagle_ctx *ctx, int on);
+int peagle_timing_read(peagle_ctx *ctx, double *ms_out, int64_t *n_out);
 
 /*
  * Forward of one query partition (Section 3; Algorithm 1 supplies the partition).

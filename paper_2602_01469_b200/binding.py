@@ -25,6 +25,7 @@ EXPORTS = [
     "peagle_tile_shape", "peagle_poll_status", "peagle_launch_count", "peagle_attn_fwd",
     "peagle_attn_bwd", "peagle_attn_partitioned", "peagle_attn_partitioned_host",
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
+    "peagle_timing_enable", "peagle_timing_read",
 ]
 
 
@@ -174,6 +175,18 @@ def peagle_poll_status(ctx: Context, stream=None) -> int:
 
 def peagle_launch_count(ctx: Context) -> int:
     return int(lib().peagle_launch_count(ctx.h))
+
+
+def peagle_timing_enable(ctx: Context, on: bool):
+    _check(lib().peagle_timing_enable(ctx.h, int(bool(on))))
+
+
+def peagle_timing_read(ctx: Context):
+    """((forward ms, backward ms), (forward launches, backward launches)) since the last read."""
+    ms = (ctypes.c_double * 2)()
+    n = (ctypes.c_int64 * 2)()
+    _check(lib().peagle_timing_read(ctx.h, ms, n), ctx.h)
+    return (ms[0], ms[1]), (n[0], n[1])
 
 
 def peagle_attn_fwd(ctx, prob: Problem, part: Partition, Q, K, V, O, LSE, stream=None):

@@ -22,6 +22,9 @@ struct peagle_ctx {
     DevBuf plan_buf, bwd_buf, acc_buf, host_buf;
     int64_t launches = 0;
     char cuda_err[256] = {0};
+    bool timing = false;
+    std::vector<cudaEvent_t> ev[2]; // recorded (start, stop) pairs: [0] forward, [1] backward
+    size_t ev_used[2] = {0, 0};
 };
 
 namespace {
@@ -60,6 +63,24 @@ int ensure(peagle_ctx *ctx, DevBuf &b, size_t bytes, cudaStream_t s)
     }
     b.bytes = want;
     return PEAGLE_OK;
+}
+
+// Next (start, stop) event pair of a kind, or nulls when timing is off or the pool is full.
+void next_events(peagle_ctx *ctx, int kind, cudaEvent_t *e0, cudaEvent_t *e1)
+{
+    *e0 = *e1 = nullptr;
+    if (!ctx->timing || ctx->ev_used[kind] >= 2 * 4096)
+        return;
+    std::vector<cudaEvent_t> &v = ctx->ev[kind];
+    while (v.size() < ctx->ev_used[kind] + 2) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess)
+            return;
+        v.push_back(e);
+    }
+    *e0 = v[ctx->ev_used[kind]];
+    *e1 = v[ctx->ev_used[kind] + 1];
+    ctx->ev_used[kind] += 2;
 }
 
 struct Carver {
@@ -213,7 +234,9 @@ int run_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
     a.Hkv = prob->n_kv_heads;
     a.D = prob->head_dim;
     a.scale = prob->softmax_scale;
-    const int n = launch_fwd(c.plan, a, ctx->encode, ctx->n_sm, s);
+    cudaEvent_t e0, e1;
+    next_events(ctx, 0, &e0, &e1);
+    const int n = launch_fwd(c.plan, a, ctx->encode, ctx->n_sm, s, e0, e1);
     if (n < 0)
         return n;
     ctx->launches += n;
@@ -250,7 +273,9 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
     a.Hkv = prob->n_kv_heads;
     a.D = prob->head_dim;
     a.scale = prob->softmax_scale;
-    const int n = launch_bwd(c.plan, a, ctx->encode, ctx->n_sm, s);
+    cudaEvent_t e0, e1;
+    next_events(ctx, 1, &e0, &e1);
+    const int n = launch_bwd(c.plan, a, ctx->encode, ctx->n_sm, s, e0, e1);
     if (n < 0)
         return n;
     ctx->launches += n;
@@ -310,6 +335,9 @@ int peagle_destroy(peagle_ctx *ctx)
             cudaFree(b->ptr);
     if (ctx->status)
         cudaFree(ctx->status);
+    for (int k = 0; k < 2; ++k)
+        for (cudaEvent_t e : ctx->ev[k])
+            cudaEventDestroy(e);
     delete ctx;
     return PEAGLE_OK;
 }
@@ -360,6 +388,34 @@ int peagle_poll_status(peagle_ctx *ctx, void *stream)
 }
 
 int64_t peagle_launch_count(const peagle_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int peagle_timing_enable(peagle_ctx *ctx, int on)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    ctx->timing = on != 0;
+    return PEAGLE_OK;
+}
+
+int peagle_timing_read(peagle_ctx *ctx, double *ms_out, int64_t *n_out)
+{
+    if (!ctx || !ms_out || !n_out)
+        return PEAGLE_ERR_NULL;
+    CK(cudaSetDevice(ctx->device));
+    CK(cudaDeviceSynchronize());
+    for (int k = 0; k < 2; ++k) {
+        double total = 0.0;
+        for (size_t i = 0; i + 1 < ctx->ev_used[k]; i += 2) {
+            float ms = 0.f;
+            CK(cudaEventElapsedTime(&ms, ctx->ev[k][i], ctx->ev[k][i + 1]));
+            total += ms;
+        }
+        ms_out[k] = total;
+        n_out[k] = (int64_t)(ctx->ev_used[k] / 2);
+        ctx->ev_used[k] = 0;
+    }
+    return PEAGLE_OK;
+}
 
 int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
                     const void *Q, const void *K, const void *V, void *O, float *LSE, void *stream)

@@ -509,7 +509,8 @@ __global__ void cast_grads_kernel(const float *__restrict__ a, const float *__re
 }
 
 template <int D>
-static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
+                        cudaEvent_t ev0, cudaEvent_t ev1)
 {
     // Q and dO maps end at the partition's last row so that rows past it read as zeros.
     CUtensorMap tmQ, tmdO, tmK, tmV;
@@ -550,7 +551,11 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
                 return PEAGLE_ERR_CUDA;
             attr_set = true;
         }
+        if (ev0)
+            cudaEventRecord(ev0, s);
         bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+        if (ev1)
+            cudaEventRecord(ev1, s);
         ++launches;
     }
     bwd_finish_dq<<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
@@ -558,11 +563,13 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
     return launches + 1;
 }
 
-int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
+               cudaEvent_t ev0, cudaEvent_t ev1)
 {
     if (p.n_qt == 0)
         return 0;
-    return a.D == 64 ? launch_bwd_t<64>(p, a, enc, n_sm, s) : launch_bwd_t<128>(p, a, enc, n_sm, s);
+    return a.D == 64 ? launch_bwd_t<64>(p, a, enc, n_sm, s, ev0, ev1)
+                     : launch_bwd_t<128>(p, a, enc, n_sm, s, ev0, ev1);
 }
 
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,

@@ -383,7 +383,8 @@ int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, in
 }
 
 template <int D>
-static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cudaStream_t s)
+static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cudaStream_t s,
+                        cudaEvent_t ev0, cudaEvent_t ev1)
 {
     CUtensorMap tmQ, tmK, tmV;
     if (make_map(enc, &tmQ, a.Q, D, a.Hq, p.T) || make_map(enc, &tmK, a.K, D, a.Hkv, p.T) ||
@@ -413,16 +414,22 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
         attr_set = true;
     }
     const int n_hb = P.two ? a.Hq / 2 : a.Hq;
+    if (ev0)
+        cudaEventRecord(ev0, s);
     fwd_kernel<D><<<p.n_qt * n_hb, 320, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
+    if (ev1)
+        cudaEventRecord(ev1, s);
     return 1;
 }
 
-int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s)
+int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
+               cudaEvent_t ev0, cudaEvent_t ev1)
 {
     (void)n_sm;
     if (p.n_qt == 0)
         return 0;
-    return a.D == 64 ? launch_fwd_t<64>(p, a, enc, s) : launch_fwd_t<128>(p, a, enc, s);
+    return a.D == 64 ? launch_fwd_t<64>(p, a, enc, s, ev0, ev1)
+                     : launch_fwd_t<128>(p, a, enc, s, ev0, ev1);
 }
 
 } // namespace peagle

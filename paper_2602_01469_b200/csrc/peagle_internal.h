@@ -76,8 +76,11 @@ int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int 
 int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s);
 
 // K1 / K2.  Return the number of kernels launched, or a negative peagle_status.
-int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s);
-int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s);
+// ev0/ev1 (may be null) are recorded on the stream right before / after the main kernel.
+int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
+               cudaEvent_t ev0, cudaEvent_t ev1);
+int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
+               cudaEvent_t ev0, cudaEvent_t ev1);
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s);
 

@@ -60,6 +60,8 @@ WORKLOADS = {
     "longtail_varlen": Workload("longtail_varlen", longtail_lengths(), 8, 64, 8, 64,
                                 seg_len=8192, seed=50),
 }
+# a half-length copy of the headline shape, small enough for profiler captures
+WORKLOADS["gptoss_n2048_profile"] = Workload("gptoss_n2048_profile", (2048,), 8, 64, 8, 64, seed=31)
 HEADLINE = "gptoss_n4096"
 
 
@@ -155,8 +157,3 @@ def build_case(w: Workload, assign_fn):
     return (np.asarray(cu, np.int32), np.concatenate(anchors).astype(np.int32),
             np.concatenate(depths).astype(np.int32), parts)
 
-
-def allowed_pairs_full_grid(n: int, K: int) -> int:
-    """Number of (query, key) pairs the mask allows on a full grid: a token at position
-    anchor+depth sees anchor+1 real tokens and `depth` chain tokens."""
-    return K * n * (n + 1) // 2 + n * K * (K - 1) // 2
