@@ -227,6 +227,9 @@ int peagle_oracle_attn_fwd(int T, const int32_t *anchor, const int32_t *depth, i
  * dQ is [nrows][h_end-h_begin][D] (overwritten).  dK, dV are [T][Hkv][D] and are ADDED to, so a
  * caller can sum the contributions of several query partitions (within-sequence gradient
  * accumulation, Section 3.2).
+ *
+ * Two sweeps: the first goes row by row (LSE, Delta and dQ of each row); the second goes key by
+ * key and sums that key's dK, dV over the listed rows, so no two threads write the same place.
  */
 int peagle_oracle_attn_bwd(int T, const int32_t *anchor, const int32_t *depth, int Hq, int Hkv,
                            int D, double scale, const int32_t *kranges, int nk,
@@ -237,19 +240,20 @@ int peagle_oracle_attn_bwd(int T, const int32_t *anchor, const int32_t *depth, i
     if (Hq % Hkv != 0 || h_begin < 0 || h_end > Hq || h_begin > h_end)
         return -1;
     const int G = Hq / Hkv, HS = h_end - h_begin;
-    for (int h = h_begin; h < h_end; ++h) {
-        const int g = h / G;
+    double *LSE = (double *)malloc(sizeof(double) * (size_t)(nrows > 0 ? nrows : 1) * (HS > 0 ? HS : 1));
+    double *DEL = (double *)malloc(sizeof(double) * (size_t)(nrows > 0 ? nrows : 1) * (HS > 0 ? HS : 1));
+    /* ---- sweep 1: per row: LSE, O, Delta, dQ */
 #pragma omp parallel
-        {
-            uint8_t *m = (uint8_t *)malloc((size_t)T);
-            double *s = (double *)malloc(sizeof(double) * (size_t)T);
-            double *dKp = (double *)calloc((size_t)T * D, sizeof(double));
-            double *dVp = (double *)calloc((size_t)T * D, sizeof(double));
-            double *o = (double *)malloc(sizeof(double) * (size_t)D);
+    {
+        uint8_t *m = (uint8_t *)malloc((size_t)T);
+        double *s = (double *)malloc(sizeof(double) * (size_t)T);
+        double *o = (double *)malloc(sizeof(double) * (size_t)D);
 #pragma omp for schedule(dynamic, 4)
-            for (int r = 0; r < nrows; ++r) {
-                const int q = rows[r];
-                mask_row(T, anchor, depth, kranges, nk, q, m);
+        for (int r = 0; r < nrows; ++r) {
+            const int q = rows[r];
+            mask_row(T, anchor, depth, kranges, nk, q, m);
+            for (int h = h_begin; h < h_end; ++h) {
+                const int g = h / G;
                 const float *qv = Q + ((size_t)q * Hq + h) * D;
                 const float *gov = dO + ((size_t)q * Hq + h) * D;
                 double *dq = dQ + ((size_t)r * HS + (h - h_begin)) * D;
@@ -267,6 +271,8 @@ int peagle_oracle_attn_bwd(int T, const int32_t *anchor, const int32_t *depth, i
                     if (s[k] > smax)
                         smax = s[k];
                 }
+                LSE[(size_t)r * HS + (h - h_begin)] = -INFINITY;
+                DEL[(size_t)r * HS + (h - h_begin)] = 0.0;
                 if (smax == -INFINITY)
                     continue;
                 double denom = 0.0;
@@ -297,27 +303,52 @@ int peagle_oracle_attn_bwd(int T, const int32_t *anchor, const int32_t *depth, i
                     for (int d = 0; d < D; ++d)
                         dp += (double)gov[d] * (double)vv[d];
                     const double ds = p * (dp - delta);
-                    for (int d = 0; d < D; ++d) {
+                    for (int d = 0; d < D; ++d)
                         dq[d] += scale * ds * (double)kv[d];
-                        dKp[(size_t)k * D + d] += scale * ds * (double)qv[d];
-                        dVp[(size_t)k * D + d] += p * (double)gov[d];
-                    }
+                }
+                LSE[(size_t)r * HS + (h - h_begin)] = lse;
+                DEL[(size_t)r * HS + (h - h_begin)] = delta;
+            }
+        }
+        free(m);
+        free(s);
+        free(o);
+    }
+    /* ---- sweep 2: per key: dK, dV summed over the listed rows and the heads of its group */
+#pragma omp parallel for schedule(dynamic, 8)
+    for (int k = 0; k < T; ++k) {
+        if (!visible(k, kranges, nk))
+            continue;
+        for (int r = 0; r < nrows; ++r) {
+            const int q = rows[r];
+            if (!peagle_oracle_allowed(anchor[q], depth[q], anchor[k], depth[k]))
+                continue;
+            for (int h = h_begin; h < h_end; ++h) {
+                const double lse = LSE[(size_t)r * HS + (h - h_begin)];
+                if (lse == -INFINITY)
+                    continue;
+                const int g = h / G;
+                const float *qv = Q + ((size_t)q * Hq + h) * D;
+                const float *gov = dO + ((size_t)q * Hq + h) * D;
+                const float *kv = K + ((size_t)k * Hkv + g) * D;
+                const float *vv = V + ((size_t)k * Hkv + g) * D;
+                double acc = 0.0, dp = 0.0;
+                for (int d = 0; d < D; ++d) {
+                    acc += (double)qv[d] * (double)kv[d];
+                    dp += (double)gov[d] * (double)vv[d];
+                }
+                const double p = exp(scale * acc - lse);
+                const double ds = p * (dp - DEL[(size_t)r * HS + (h - h_begin)]);
+                double *dk = dK + ((size_t)k * Hkv + g) * D;
+                double *dv = dV + ((size_t)k * Hkv + g) * D;
+                for (int d = 0; d < D; ++d) {
+                    dk[d] += scale * ds * (double)qv[d];
+                    dv[d] += p * (double)gov[d];
                 }
             }
-#pragma omp critical
-            {
-                for (int k = 0; k < T; ++k)
-                    for (int d = 0; d < D; ++d) {
-                        dK[((size_t)k * Hkv + g) * D + d] += dKp[(size_t)k * D + d];
-                        dV[((size_t)k * Hkv + g) * D + d] += dVp[(size_t)k * D + d];
-                    }
-            }
-            free(m);
-            free(s);
-            free(dKp);
-            free(dVp);
-            free(o);
         }
     }
+    free(LSE);
+    free(DEL);
     return 0;
 }
