@@ -123,6 +123,46 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
                     const void *Q, const void *K, const void *V, void *O, float *LSE, void *stream);
 
 /*
+ * Forward of one query partition for callers that must not allocate device memory.  (The paper
+ * has no counterpart: this is a packaging variant of peagle_attn_fwd, same arithmetic, same
+ * kernels.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a training step inside a
+ * framework whose caching allocator already owns nearly all of the GPU's memory (a raw
+ * allocation there fails or makes the framework give its cache back), a latency-critical loop
+ * that cannot afford the device-wide synchronisation an allocation implies, or a plug-in host
+ * that forbids allocation in its execute callback.  peagle_attn_fwd keeps the tile plan of a
+ * call (packed metadata, tile classes, work lists) in context scratch that grows with
+ * cudaMalloc; this entry point needs no context and keeps the plan in a fixed array that is
+ * part of the library image instead.  It calls no cudaMalloc, cudaFree or any routine that
+ * allocates.
+ *
+ * Cost and limits: the array is PEAGLE_STATIC_SCRATCH_BYTES (2 MiB) of device memory on every
+ * GPU that loads the library, held until the process exits.  Accepted sizes:
+ * prob->total_tokens <= PEAGLE_STATIC_MAX_TOKENS and (query tiles of the partition) x (key tiles
+ * of its visible ranges) <= PEAGLE_STATIC_MAX_TILE_PAIRS, tiles as peagle_tile_shape reports
+ * them; anything larger returns PEAGLE_ERR_TOO_LARGE and launches nothing.
+ *
+ * `device` is the CUDA device ordinal (made current by the call).  The first call on a device
+ * looks up the array's device address and the tensor-map encoder, once; make that first call
+ * before any stream capture begins.  Work is enqueued on `stream` and the call returns without
+ * waiting.  `dev_status` (dev, may be NULL) is one int32 owned by the caller: the call clears it
+ * on the stream, and a device-side error (PEAGLE_ERR_BAD_META, PEAGLE_ERR_TIMEOUT) is written
+ * there; read it after synchronising the stream.
+ *
+ * All calls on a device share the one array, and it keeps the previous call's contents (the
+ * call re-initialises everything it reads).  Two calls whose GPU work overlaps -- different
+ * streams, or different host threads -- race on it: keep them on one stream or order them with
+ * events.  Q, K, V, O, LSE, prob and part exactly as for peagle_attn_fwd.
+ */
+#define PEAGLE_STATIC_SCRATCH_BYTES (2u << 20)
+#define PEAGLE_STATIC_MAX_TOKENS 32768
+#define PEAGLE_STATIC_MAX_TILE_PAIRS 65536
+int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,
+                           const peagle_partition_t *part, const void *Q, const void *K,
+                           const void *V, void *O, float *LSE, int32_t *dev_status, void *stream);
+
+/*
  * Backward of one query partition (Section 3.2: one forward-backward per segment, gradients
  * accumulated across the segments of a sequence).  With P = exp(s - LSE), Delta = <dO, O>,
  * dP_k = <dO[q,h], V[k,g]>, dS_k = P_k (dP_k - Delta):

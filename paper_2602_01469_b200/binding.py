@@ -25,7 +25,7 @@ EXPORTS = [
     "peagle_tile_shape", "peagle_poll_status", "peagle_launch_count", "peagle_attn_fwd",
     "peagle_attn_bwd", "peagle_attn_partitioned", "peagle_attn_partitioned_host",
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
-    "peagle_timing_enable", "peagle_timing_read",
+    "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
 ]
 
 
@@ -192,6 +192,16 @@ def peagle_timing_read(ctx: Context):
 def peagle_attn_fwd(ctx, prob: Problem, part: Partition, Q, K, V, O, LSE, stream=None):
     _check(lib().peagle_attn_fwd(ctx.h, prob.ref(), part.ref(), _ptr(Q), _ptr(K), _ptr(V), _ptr(O),
                                  _ptr(LSE), _stream(stream)), ctx.h)
+
+
+def peagle_attn_fwd_static(device: int, prob: Problem, part: Partition, Q, K, V, O, LSE,
+                           dev_status=None, stream=None):
+    """Forward without any device allocation: the call's tile plan lives in a fixed array inside
+    the library (2 MiB per GPU), so no context is needed.  ``dev_status`` is an optional int32
+    device tensor that receives a device-side error code."""
+    _check(lib().peagle_attn_fwd_static(int(device), prob.ref(), part.ref(), _ptr(Q), _ptr(K),
+                                        _ptr(V), _ptr(O), _ptr(LSE), _ptr(dev_status),
+                                        _stream(stream)))
 
 
 def peagle_attn_bwd(ctx, prob: Problem, part: Partition, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc,

@@ -3,6 +3,7 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
 #include <vector>
 
 #include "peagle_internal.h"
@@ -285,6 +286,65 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
 
 } // namespace
 
+// ---- scratch of peagle_attn_fwd_static ------------------------------------------------------
+// Lives in the library image: every GPU that loads the library holds these bytes until the
+// process exits.  Layout: the K0 plan (carve_plan) from byte 0, a fallback status word in the
+// last 256 bytes.
+constexpr size_t STATIC_SCRATCH_BYTES = size_t(2) << 20;
+constexpr int STATIC_MAX_TOKENS = 32768;
+constexpr int STATIC_MAX_TILE_PAIRS = 65536;
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+namespace {
+
+struct StaticDevice {
+    bool ready = false;
+    unsigned char *scratch = nullptr; // device address of g_static_scratch on this device
+    EncodeTiledFn encode = nullptr;
+    int n_sm = 0;
+};
+constexpr int STATIC_MAX_DEVICES = 64;
+StaticDevice g_static_dev[STATIC_MAX_DEVICES];
+std::mutex g_static_mutex;
+
+// One-time set-up of a device for peagle_attn_fwd_static; `device` is current.  In host code
+// `g_static_scratch` is only a handle for the runtime, so the array's real device address is
+// looked up here and that pointer is what the kernels get.
+int static_setup(int device, StaticDevice **out)
+{
+    if (device < 0 || device >= STATIC_MAX_DEVICES)
+        return PEAGLE_ERR_TOO_LARGE;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDevice &d = g_static_dev[device];
+    if (!d.ready) {
+        int major = 0, n_sm = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        if (major != 10)
+            return PEAGLE_ERR_UNSUPPORTED_ARCH;
+        void *addr = nullptr;
+        if (cudaGetSymbolAddress((void **)&addr, g_static_scratch) != cudaSuccess || !addr) {
+            cudaGetLastError();
+            return PEAGLE_ERR_CUDA;
+        }
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) !=
+                cudaSuccess ||
+            qres != cudaDriverEntryPointSuccess || !fn)
+            return PEAGLE_ERR_CUDA;
+        d.scratch = static_cast<unsigned char *>(addr);
+        d.encode = reinterpret_cast<EncodeTiledFn>(fn);
+        d.n_sm = n_sm;
+        d.ready = true;
+    }
+    *out = &d;
+    return PEAGLE_OK;
+}
+
+} // namespace
+
 extern "C" {
 
 int peagle_create(peagle_ctx **out, int device)
@@ -434,6 +494,73 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
     if (rc != PEAGLE_OK)
         return rc;
     return run_fwd(ctx, prob, c, Q, K, V, O, LSE, s);
+}
+
+int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,
+                           const peagle_partition_t *part, const void *Q, const void *K,
+                           const void *V, void *O, float *LSE, int32_t *dev_status, void *stream)
+{
+    if (!Q || !K || !V || !O || !LSE)
+        return PEAGLE_ERR_NULL;
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O))
+        return PEAGLE_ERR_ALIGN;
+    Call c;
+    rc = validate_partition(prob, part, c);
+    if (rc != PEAGLE_OK)
+        return rc;
+    // The limits are checked before anything touches the device.
+    if (prob->total_tokens > STATIC_MAX_TOKENS ||
+        (int64_t)c.plan.n_qt * (int64_t)c.plan.n_kt > STATIC_MAX_TILE_PAIRS)
+        return PEAGLE_ERR_TOO_LARGE;
+    size_t plan_bytes = 0;
+    carve_plan(c.plan, nullptr, &plan_bytes);
+    if (plan_bytes + 256 > STATIC_SCRATCH_BYTES)
+        return PEAGLE_ERR_TOO_LARGE;
+    if (cudaSetDevice(device) != cudaSuccess) {
+        cudaGetLastError();
+        return PEAGLE_ERR_CUDA;
+    }
+    StaticDevice *dev = nullptr;
+    rc = static_setup(device, &dev);
+    if (rc != PEAGLE_OK)
+        return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    carve_plan(c.plan, dev->scratch, nullptr);
+    int *status = dev_status ? dev_status
+                             : reinterpret_cast<int *>(dev->scratch + STATIC_SCRATCH_BYTES - 256);
+    c.plan.status = status;
+    // The array keeps whatever the previous call left.  The status word is cleared here; the
+    // plan's counters are cleared by the first K0 kernel; every other plan field this call
+    // reads is written by this call's K0 kernels first.
+    if (cudaMemsetAsync(status, 0, sizeof(int), s) != cudaSuccess) {
+        cudaGetLastError();
+        return PEAGLE_ERR_CUDA;
+    }
+    if (c.plan.n_qt == 0)
+        return PEAGLE_OK;
+    launch_plan(c.plan, prob->anchor, prob->depth, prob->K, c.seq_begin, c.seq_end, c.ranges,
+                false, prob->n_kv_heads, s);
+    if (cudaGetLastError() != cudaSuccess)
+        return PEAGLE_ERR_CUDA;
+    FwdArgs a;
+    a.Q = Q;
+    a.K = K;
+    a.V = V;
+    a.O = O;
+    a.LSE = LSE;
+    a.Hq = prob->n_q_heads;
+    a.Hkv = prob->n_kv_heads;
+    a.D = prob->head_dim;
+    a.scale = prob->softmax_scale;
+    const int n = launch_fwd(c.plan, a, dev->encode, dev->n_sm, s, nullptr, nullptr);
+    if (n < 0)
+        return n;
+    if (cudaGetLastError() != cudaSuccess)
+        return PEAGLE_ERR_CUDA;
+    return PEAGLE_OK;
 }
 
 int peagle_attn_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
