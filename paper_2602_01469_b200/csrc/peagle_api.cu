@@ -112,9 +112,10 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.klist = c.take<int2>(nq * nk);
     p.kcount = c.take<int>(nq);
     p.qorder = c.take<int>(nq);
-    p.qlist = c.take<int2>(nq * nk);
-    p.qcount = c.take<int>(nk);
-    p.bitems = c.take<int4>(nk * ((nq + BWD_CQ - 1) / BWD_CQ));
+    const size_t nch = (nq + BWD_CQ - 1) / BWD_CQ;
+    p.cmask = c.take<uint16_t>(nch * nk);
+    p.ccount = c.take<int>(nch);
+    p.bitems = c.take<int4>(nch * nk);
     if (bytes_out)
         *bytes_out = c.off + 256;
 }

@@ -28,7 +28,6 @@ int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, in
 
 struct BwdParams {
     const int2 *ktile;
-    const int2 *qlist;
     const int4 *bitems;
     const int *counters;
     const int32_t *meta;
@@ -151,8 +150,8 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
             }
             ok = __all_sync(0xffffffffu, ok);
-            for (int e = 0; ok && e < item.z; ++e) {
-                const int qt = P.qlist[(size_t)kt * P.n_qt + item.y + e].x;
+            for (unsigned em = (unsigned)item.z & 0xffu; ok && em; em &= em - 1) {
+                const int qt = item.y * BWD_CQ + (__ffs(em) - 1);
                 const int row0 = P.q_begin + qt * BM;
                 for (int hh = 0; ok && hh < G; ++hh, ++it) {
                     const int h = g * G + hh;
@@ -203,7 +202,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             bool ok = true;
             for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
                 const int4 item = P.bitems[idx / P.Hkv];
-                const int n_it = item.z * G;
+                const int n_it = item.w * G;
                 ok = mbar_wait(BAR(B_KVFULL), w & 1, abort_flag) &&
                      mbar_wait(BAR(B_ACCFREE), (w & 1) ^ 1, abort_flag);
                 for (int i = 0; ok && i < n_it; ++i, ++it) {
@@ -285,10 +284,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             const int kt = item.x;
             const int2 ktile = P.ktile[kt];
             const int32_t mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
-            for (int e = 0; ok && e < item.z; ++e) {
-                const int2 qe = P.qlist[(size_t)kt * P.n_qt + item.y + e];
-                const int row0 = P.q_begin + qe.x * BM;
-                const bool full = qe.y == TILE_FULL;
+            for (unsigned em = (unsigned)item.z & 0xffu; ok && em; em &= em - 1) {
+                const int eb = __ffs(em) - 1;
+                const int row0 = P.q_begin + (item.y * BWD_CQ + eb) * BM;
+                const bool full = ((unsigned)item.z >> (8 + eb)) & 1u;
                 for (int hh = 0; ok && hh < G; ++hh, ++it) {
                     const int h = g * G + hh;
                     const int st = it % NSQ, ph = (it / NSQ) & 1;
@@ -437,6 +436,482 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// head_dim 64: software-pipelined variant.  Tensor memory has room for two dQ accumulators, so the
+// MMA warp runs one step ahead of the compute warps:
+//   while the compute warps turn S^T(i) into P^T(i):   dK(i-1), dQ(i-1), dP^T(i)
+//   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
+// and dQ(i-1) is drained to the fp32 staging rows after dS^T(i) has been handed over.  K / V of
+// the next work item are prefetched into a second stage.  384 threads: warps 0-7 compute, warp 8
+// issues MMAs, warp 9 produces, warps 10-11 only give their registers to the compute warps.
+struct Bwd64Cfg {
+    static constexpr int D = 64;
+    static constexpr int NSQ = 3;
+    static constexpr int TILE_BYTES = 128 * 128;
+    static constexpr int OFF_KV = 0;                              // 2 stages x (K, V)
+    static constexpr int OFF_DS = 4 * TILE_BYTES;                 // 2 panels
+    static constexpr int OFF_Q = OFF_DS + 2 * TILE_BYTES;         // ring of (Q, dO)
+    static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (-lse2[128], -delta[128], mq[128])
+    static constexpr int ROW_BYTES = 3 * 128 * 4;
+    static constexpr int OFF_BAR = OFF_ROW + NSQ * ROW_BYTES;
+    static constexpr int N_BAR = 2 * NSQ + 13;
+    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
+    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
+    static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 256 /* two of 64 */, TM_DK = 384, TM_DV = 448;
+};
+
+// Walks the (work item, query tile, head) iterations of one CTA in execution order.
+struct BwdWalk {
+    const int4 *bitems;
+    int idx, stride, total, Hkv, G;
+    int kt, g, c, w;
+    unsigned mask, em;
+    int hh;
+    bool valid;
+    __device__ void load()
+    {
+        valid = idx < total;
+        if (!valid)
+            return;
+        const int4 item = bitems[idx / Hkv];
+        g = idx % Hkv;
+        kt = item.x;
+        c = item.y;
+        mask = (unsigned)item.z;
+        em = mask & 0xffu;
+        hh = 0;
+    }
+    __device__ void init(const BwdParams &P, int first, int step)
+    {
+        bitems = P.bitems;
+        idx = first;
+        stride = step;
+        Hkv = P.Hkv;
+        G = P.Hq / P.Hkv;
+        total = P.counters[1] * P.Hkv;
+        w = 0;
+        load();
+    }
+    __device__ bool first() const { return hh == 0 && em == (mask & 0xffu); }
+    __device__ bool last() const { return hh == G - 1 && (em & (em - 1)) == 0; }
+    __device__ int qt() const { return c * BWD_CQ + (__ffs(em) - 1); }
+    __device__ bool full() const { return (mask >> (8 + __ffs(em) - 1)) & 1u; }
+    __device__ int head() const { return g * G + hh; }
+    __device__ void next()
+    {
+        if (++hh == G) {
+            hh = 0;
+            em &= em - 1;
+            if (em == 0) {
+                idx += stride;
+                ++w;
+                load();
+            }
+        }
+    }
+};
+
+__global__ void __launch_bounds__(384, 1)
+bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
+             const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+             const BwdParams P)
+{
+    using C = Bwd64Cfg;
+    constexpr int D = 64, NSQ = C::NSQ, TB = C::TILE_BYTES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u;
+    uint8_t *sp = smem_raw + (sb - raw);
+    const uint32_t bar0 = sb + C::OFF_BAR;
+    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+    constexpr int B_QFULL = 0, B_QEMPTY = NSQ, B_KVFULL = 2 * NSQ, B_KVEMPTY = B_KVFULL + 2,
+                  B_SFULL = B_KVFULL + 4, B_DPFULL = B_KVFULL + 5, B_PFULL = B_KVFULL + 6,
+                  B_DSFULL = B_KVFULL + 7, B_DQFULL = B_KVFULL + 8, B_DQEMPTY = B_KVFULL + 10,
+                  B_ACCFREE = B_KVFULL + 12;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < NSQ; ++s) {
+            mbar_init(BAR(B_QFULL + s), 1);
+            mbar_init(BAR(B_QEMPTY + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(BAR(B_KVFULL + s), 1);
+            mbar_init(BAR(B_KVEMPTY + s), 1);
+            mbar_init(BAR(B_DQFULL + s), 1);
+            mbar_init(BAR(B_DQEMPTY + s), 256);
+        }
+        mbar_init(BAR(B_SFULL), 1);
+        mbar_init(BAR(B_DPFULL), 1);
+        mbar_init(BAR(B_PFULL), 256);
+        mbar_init(BAR(B_DSFULL), 256);
+        mbar_init(BAR(B_ACCFREE), 256);
+        fence_mbar_init();
+    }
+    if (warp == 8) {
+        tmem_alloc(sb + C::OFF_MISC, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp >= 8) {
+        reg_dec<56>();
+        if (warp == 9) {
+            // -------------------------------------------------------- producer
+            if (lane == 0) {
+                tma_prefetch_desc(&tmQ);
+                tma_prefetch_desc(&tmdO);
+                tma_prefetch_desc(&tmK);
+                tma_prefetch_desc(&tmV);
+            }
+            BwdWalk wk;
+            wk.init(P, blockIdx.x, gridDim.x);
+            auto load_kv = [&](int w, int kt, int g) -> bool {
+                bool ok = true;
+                if (lane == 0) {
+                    const int s = w & 1;
+                    ok = mbar_wait(BAR(B_KVEMPTY + s), ((w >> 1) & 1) ^ 1, abort_flag);
+                    if (ok) {
+                        const int start = P.ktile[kt].x;
+                        mbar_arrive_expect_tx(BAR(B_KVFULL + s), 2 * TB);
+                        tma_load_3d(sb + C::OFF_KV + (2 * s) * TB, &tmK, BAR(B_KVFULL + s), 0, g, start);
+                        tma_load_3d(sb + C::OFF_KV + (2 * s + 1) * TB, &tmV, BAR(B_KVFULL + s), 0, g, start);
+                    }
+                }
+                return __all_sync(0xffffffffu, ok);
+            };
+            bool ok = true;
+            if (wk.valid)
+                ok = load_kv(0, wk.kt, wk.g);
+            for (int it = 0; ok && wk.valid; ++it) {
+                const int st = it % NSQ, ph = (it / NSQ) & 1;
+                const int row0 = P.q_begin + wk.qt() * BM;
+                const int h = wk.head();
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
+                if (!ok)
+                    break;
+                float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
+                for (int i = lane; i < BM; i += 32) {
+                    const int row = row0 + i;
+                    float nl2 = -CUDART_INF_F, ndl = 0.f;
+                    int mq = META_NONE_Q;
+                    if (row < P.q_end) {
+                        const float lse = P.LSE[(size_t)h * P.T + row];
+                        if (lse != -CUDART_INF_F)
+                            nl2 = -lse * 1.4426950408889634f;
+                        ndl = -P.delta[(size_t)h * (P.q_end - P.q_begin) + (row - P.q_begin)];
+                        mq = P.meta[row];
+                        if (mq == META_NONE_K)
+                            mq = META_NONE_Q;
+                    }
+                    rowbuf[i] = nl2;
+                    rowbuf[128 + i] = ndl;
+                    reinterpret_cast<int *>(rowbuf)[256 + i] = mq;
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * TB);
+                    const uint32_t qa = sb + C::OFF_Q + st * 2 * TB;
+                    tma_load_3d(qa, &tmQ, BAR(B_QFULL + st), 0, h, row0);
+                    tma_load_3d(qa + TB, &tmdO, BAR(B_QFULL + st), 0, h, row0);
+                }
+                const bool was_last = wk.last();
+                wk.next();
+                if (was_last && wk.valid)
+                    ok = load_kv(wk.w, wk.kt, wk.g); // next item's K / V into the other stage
+            }
+        } else if (warp == 8 && lane == 0) {
+            // -------------------------------------------------------- MMA issue
+            constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
+            constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
+            constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
+            const uint32_t dsa = sb + C::OFF_DS;
+            auto issue_s = [&](uint32_t ka, uint32_t qa) {
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k)
+                    mma_ss(tmem + C::TM_S, smem_desc_sw128(ka + k * 32, 16, 1024),
+                           smem_desc_sw128(qa + k * 32, 16, 1024), IDESC_S, k > 0);
+            };
+            auto issue_dp = [&](uint32_t va, uint32_t doa) {
+#pragma unroll
+                for (int k = 0; k < D / 16; ++k)
+                    mma_ss(tmem + C::TM_DP, smem_desc_sw128(va + k * 32, 16, 1024),
+                           smem_desc_sw128(doa + k * 32, 16, 1024), IDESC_S, k > 0);
+            };
+            BwdWalk cur, nxt;
+            cur.init(P, blockIdx.x, gridDim.x);
+            nxt = cur;
+            if (nxt.valid)
+                nxt.next();
+            bool ok = true;
+            if (cur.valid) {
+                ok = mbar_wait(BAR(B_KVFULL + 0), 0, abort_flag) &&
+                     mbar_wait(BAR(B_QFULL + 0), 0, abort_flag);
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t ka = sb + C::OFF_KV, qa = sb + C::OFF_Q;
+                    issue_s(ka, qa);
+                    tc_commit(BAR(B_SFULL));
+                    issue_dp(ka + TB, qa + TB);
+                    tc_commit(BAR(B_DPFULL));
+                }
+            }
+            for (int it = 0; ok && cur.valid; ++it) {
+                const int st = it % NSQ;
+                const int ks = cur.w & 1;
+                const uint32_t ka = sb + C::OFF_KV + 2 * ks * TB;
+                const uint32_t qa = sb + C::OFF_Q + st * 2 * TB, doa = qa + TB;
+                const bool first = cur.first(), last = cur.last();
+                const int nst = (it + 1) % NSQ, nph = ((it + 1) / NSQ) & 1;
+                const int nks = nxt.valid ? (nxt.w & 1) : 0;
+                const uint32_t nka = sb + C::OFF_KV + 2 * nks * TB;
+                const uint32_t nqa = sb + C::OFF_Q + nst * 2 * TB;
+                // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
+                ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
+                if (ok && first)
+                    ok = mbar_wait(BAR(B_ACCFREE), (cur.w & 1) ^ 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    mma_ts(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                           smem_desc_sw128(doa + k * 2048, TB, 1024), IDESC_KV, !first || k > 0);
+                if (nxt.valid) {
+                    if (nxt.first())
+                        ok = mbar_wait(BAR(B_KVFULL + nks), (nxt.w >> 1) & 1, abort_flag);
+                    ok = ok && mbar_wait(BAR(B_QFULL + nst), nph, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    issue_s(nka, nqa);
+                    tc_commit(BAR(B_SFULL));
+                }
+                // ---- dK(it), dQ(it) once dS^T(it) is in shared memory, then dP^T(it+1)
+                ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag) &&
+                     mbar_wait(BAR(B_DQEMPTY + (it & 1)), ((it >> 1) & 1) ^ 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tmem + C::TM_DK, smem_desc_sw128(dsa + (k / 4) * TB + (k % 4) * 32, 16, 1024),
+                           smem_desc_sw128(qa + k * 2048, TB, 1024), IDESC_KV, !first || k > 0);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    mma_ss(tmem + C::TM_DQ + (it & 1) * 64, smem_desc_sw128(dsa + k * 2048, TB, 1024),
+                           smem_desc_sw128(ka + k * 2048, TB, 1024), IDESC_DQ, k > 0);
+                tc_commit(BAR(B_DQFULL + (it & 1)));
+                tc_commit(BAR(B_QEMPTY + st));
+                if (last)
+                    tc_commit(BAR(B_KVEMPTY + ks));
+                if (nxt.valid) {
+                    issue_dp(nka + TB, nqa + TB);
+                    tc_commit(BAR(B_DPFULL));
+                }
+                cur = nxt;
+                if (nxt.valid)
+                    nxt.next();
+            }
+        }
+    } else {
+        reg_inc<224>();
+        // ------------------------------------------------------------ compute (warps 0-7)
+        const int wg = warp >> 2;
+        const int r = threadIdx.x & 127; // key lane for S/dP/dK/dV, query row for dQ
+        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_sel + C::TM_S + wg * 64;
+        const uint32_t tDP = tmem + lane_sel + C::TM_DP + wg * 64;
+        const uint32_t tDQ = tmem + lane_sel + C::TM_DQ + wg * 32;
+        const uint32_t tACC = tmem + lane_sel + (wg == 0 ? C::TM_DK : C::TM_DV);
+        uint8_t *dsrow = sp + C::OFF_DS + wg * TB + r * 128;
+        BwdWalk wk;
+        wk.init(P, blockIdx.x, gridDim.x);
+        bool ok = true;
+        bool pending = false;   // dQ of the previous iteration still sits in tensor memory
+        int prev_row0 = 0, prev_h = 0;
+        int32_t mk = META_NONE_K;
+        int2 ktile = make_int2(0, 0);
+        // dQ(j) -> fp32 staging rows; j's accumulator is TM_DQ + (j & 1) * 64
+        auto drain_dq = [&](int j, int row0, int h) {
+            const int row = row0 + r;
+            float *dst = P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D + wg * 32;
+            uint32_t o[32];
+            tmem_ld32(tDQ + (j & 1) * 64, o);
+            tmem_wait_ld();
+            if (row < P.q_end) {
+#pragma unroll
+                for (int i = 0; i < 32; i += 4)
+                    red_add_v4(dst + i, __uint_as_float(o[i]) * P.scale,
+                               __uint_as_float(o[i + 1]) * P.scale,
+                               __uint_as_float(o[i + 2]) * P.scale,
+                               __uint_as_float(o[i + 3]) * P.scale);
+            }
+            tc_fence_before();
+            mbar_arrive(BAR(B_DQEMPTY + (j & 1)));
+        };
+        for (int it = 0; ok && wk.valid; ++it) {
+            const int st = it % NSQ, ph = (it / NSQ) & 1;
+            if (wk.first()) {
+                ktile = P.ktile[wk.kt];
+                mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
+            }
+            const int row0 = P.q_begin + wk.qt() * BM;
+            const int h = wk.head();
+            const bool full = wk.full(), last = wk.last();
+            const float *rowbuf = reinterpret_cast<const float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
+            const float4 *nl4 = reinterpret_cast<const float4 *>(rowbuf + wg * 64);
+            const float4 *nd4 = reinterpret_cast<const float4 *>(rowbuf + 128 + wg * 64);
+            const int4 *mq4 = reinterpret_cast<const int4 *>(rowbuf + 256 + wg * 64);
+            // ---- P^T
+            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL), it & 1, abort_flag) &&
+                                             mbar_wait(BAR(B_QFULL + st), ph, abort_flag));
+            if (!ok)
+                break;
+            tc_fence_after();
+            uint32_t sr[2][32];
+            tmem_ld32(tS, sr[0]);
+            tmem_ld32(tS + 32, sr[1]);
+            tmem_wait_ld();
+            float p[64];
+#pragma unroll
+            for (int c = 0; c < 64; c += 4) {
+                const float4 l = nl4[c >> 2];
+                float a0, a1, a2, a3;
+                fma2(a0, a1, __uint_as_float(sr[c >> 5][(c + 0) & 31]),
+                     __uint_as_float(sr[c >> 5][(c + 1) & 31]), P.scale_log2, P.scale_log2, l.x, l.y);
+                fma2(a2, a3, __uint_as_float(sr[c >> 5][(c + 2) & 31]),
+                     __uint_as_float(sr[c >> 5][(c + 3) & 31]), P.scale_log2, P.scale_log2, l.z, l.w);
+                p[c + 0] = fast_exp2(a0);
+                p[c + 1] = fast_exp2(a1);
+                p[c + 2] = fast_exp2(a2);
+                p[c + 3] = fast_exp2(a3);
+            }
+            if (!full) {
+#pragma unroll
+                for (int c = 0; c < 64; c += 4) {
+                    const int4 mq = mq4[c >> 2];
+                    if (!allowed_packed(mq.x, mk)) p[c + 0] = 0.f;
+                    if (!allowed_packed(mq.y, mk)) p[c + 1] = 0.f;
+                    if (!allowed_packed(mq.z, mk)) p[c + 2] = 0.f;
+                    if (!allowed_packed(mq.w, mk)) p[c + 3] = 0.f;
+                }
+            }
+            {
+                uint32_t pk[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    pk[i] = pack_bf16x2(p[2 * i], p[2 * i + 1]);
+                tmem_st32(tS, pk); // packed P^T over the first half of this group's S^T columns
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(BAR(B_PFULL));
+            // ---- dS^T
+            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DPFULL), it & 1, abort_flag));
+            if (!ok)
+                break;
+            tc_fence_after();
+            tmem_ld32(tDP, sr[0]);
+            tmem_ld32(tDP + 32, sr[1]);
+            tmem_wait_ld();
+            tc_fence_before();
+            uint4 dsv[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) { // 16-byte chunk j = query columns 8j .. 8j+7
+                const float4 d0 = nd4[2 * j], d1 = nd4[2 * j + 1];
+                const int c = 8 * j;
+                float t0, t1, t2, t3, t4, t5, t6, t7;
+                add2(t0, t1, __uint_as_float(sr[c >> 5][(c + 0) & 31]), __uint_as_float(sr[c >> 5][(c + 1) & 31]), d0.x, d0.y);
+                add2(t2, t3, __uint_as_float(sr[c >> 5][(c + 2) & 31]), __uint_as_float(sr[c >> 5][(c + 3) & 31]), d0.z, d0.w);
+                add2(t4, t5, __uint_as_float(sr[c >> 5][(c + 4) & 31]), __uint_as_float(sr[c >> 5][(c + 5) & 31]), d1.x, d1.y);
+                add2(t6, t7, __uint_as_float(sr[c >> 5][(c + 6) & 31]), __uint_as_float(sr[c >> 5][(c + 7) & 31]), d1.z, d1.w);
+                mul2(t0, t1, t0, t1, p[c + 0], p[c + 1]);
+                mul2(t2, t3, t2, t3, p[c + 2], p[c + 3]);
+                mul2(t4, t5, t4, t5, p[c + 4], p[c + 5]);
+                mul2(t6, t7, t6, t7, p[c + 6], p[c + 7]);
+                dsv[j].x = pack_bf16x2(t0, t1);
+                dsv[j].y = pack_bf16x2(t2, t3);
+                dsv[j].z = pack_bf16x2(t4, t5);
+                dsv[j].w = pack_bf16x2(t6, t7);
+            }
+            // the dS^T buffer is free once dK / dQ of the previous iteration have run
+            if (it > 0) {
+                ok = __all_sync(0xffffffffu,
+                                mbar_wait(BAR(B_DQFULL + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag));
+                if (!ok)
+                    break;
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = dsv[j];
+            fence_proxy_async_smem();
+            mbar_arrive(BAR(B_DSFULL));
+            // ---- dQ of the previous iteration (its MMAs are done: waited on above)
+            if (pending) {
+                tc_fence_after();
+                drain_dq(it - 1, prev_row0, prev_h);
+                pending = false;
+            }
+            if (last) {
+                // end of the work item: dQ of this iteration, then dK (group 0) / dV (group 1)
+                ok = __all_sync(0xffffffffu,
+                                mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag));
+                if (!ok)
+                    break;
+                tc_fence_after();
+                drain_dq(it, row0, h);
+                float *acc = (wg == 0 ? P.dK_acc : P.dV_acc) + ((size_t)(ktile.x + r) * P.Hkv + wk.g) * D;
+                const float f = (wg == 0) ? P.scale : 1.f;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tACC + c * 32, o);
+                    tmem_wait_ld();
+                    if (r < ktile.y) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            red_add_v4(acc + c * 32 + i, __uint_as_float(o[i]) * f,
+                                       __uint_as_float(o[i + 1]) * f, __uint_as_float(o[i + 2]) * f,
+                                       __uint_as_float(o[i + 3]) * f);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(BAR(B_ACCFREE));
+            } else {
+                pending = true;
+                prev_row0 = row0;
+                prev_h = h;
+            }
+            wk.next();
+        }
+    }
+
+    // ------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {
+        }
+        __syncthreads();
+    }
+    if (warp == 8) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, 512);
+    }
+}
+
 // Delta[h][r] = <dO[q,h,:], O[q,h,:]> for the rows of the partition, and zero the fp32 dQ staging.
 template <int D>
 __global__ void bwd_prepare(const __nv_bfloat16 *__restrict__ O, const __nv_bfloat16 *__restrict__ dO,
@@ -526,7 +1001,6 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
     if (p.n_kt > 0) {
         BwdParams P;
         P.ktile = p.ktile;
-        P.qlist = p.qlist;
         P.bitems = p.bitems;
         P.counters = p.counters;
         P.meta = p.meta;
@@ -546,14 +1020,21 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         P.scale_log2 = a.scale * 1.4426950408889634f;
         static bool attr_set = false;
         if (!attr_set) {
-            if (cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     BwdCfg<D>::SMEM_BYTES) != cudaSuccess)
+            const cudaError_t e =
+                (D == 64) ? cudaFuncSetAttribute(bwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 Bwd64Cfg::SMEM_BYTES)
+                          : cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 BwdCfg<D>::SMEM_BYTES);
+            if (e != cudaSuccess)
                 return PEAGLE_ERR_CUDA;
             attr_set = true;
         }
         if (ev0)
             cudaEventRecord(ev0, s);
-        bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+        if (D == 64)
+            bwd64_kernel<<<n_sm, 384, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+        else
+            bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
         if (ev1)
             cudaEventRecord(ev1, s);
         ++launches;

@@ -11,7 +11,7 @@ namespace peagle {
 constexpr int BM = 128;          // query rows per tile
 constexpr int BN = 128;          // keys per tile
 constexpr int MAX_KRANGES = 32;  // visible key ranges per partition
-constexpr int BWD_CQ = 8;        // query tiles per backward work item
+constexpr int BWD_CQ = 8;        // query tiles per backward work item (aligned chunk; at most 8)
 constexpr int32_t META_NONE_Q = -1;         // packed metadata of a row outside the partition (sees nothing)
 constexpr int32_t META_NONE_K = 0x7fffffff; // packed metadata of a key outside the batch (seen by nobody)
 
@@ -40,9 +40,9 @@ struct Plan {
     int2 *klist;           // [n_qt][n_kt] compact non-skip key tiles per query tile: (first token, len | cls<<16)
     int *kcount;           // [n_qt]
     int *qorder;           // [n_qt] query tiles, most key tiles first
-    int2 *qlist;           // [n_kt][n_qt] compact non-skip query tiles per key tile: (qt, cls)
-    int *qcount;           // [n_kt]
-    int4 *bitems;          // [n_kt * ceil(n_qt/BWD_CQ)] backward work items (kt, first list entry, n entries, -)
+    uint16_t *cmask;       // [n_ch][n_kt] per chunk of BWD_CQ query tiles: bit b not skipped, bit 8+b FULL
+    int *ccount;           // [n_ch] key tiles with a non-zero word
+    int4 *bitems;          // [n_ch * n_kt] backward work items (key tile, chunk, mask word, query tiles)
     int *status;           // device status word
 };
 

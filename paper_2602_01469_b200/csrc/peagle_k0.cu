@@ -7,8 +7,8 @@
 //   2. summarise every query tile and key tile (min/max anchor and depth),
 //   3. classify every (query tile, key tile) pair as SKIP / PARTIAL / FULL -- from the summaries
 //      where they decide, else exactly by evaluating the predicate on the tile,
-//   4. compact the non-skipped tiles into per-query-tile lists (forward) and per-key-tile lists
-//      (backward), order query tiles longest-first and cut the backward into work items.
+//   4. compact the non-skipped tiles into per-query-tile key lists, order query tiles
+//      longest-first, and cut the backward into (key tile, query-tile chunk) work items.
 // Everything runs on the caller's stream; nothing returns to the host.
 #include "peagle_internal.h"
 
@@ -162,25 +162,20 @@ __global__ void k0_classify_exact(Plan p)
 }
 
 // ---- 4a. compact lists -------------------------------------------------------------------
-// Blocks [0, n_qt): key-tile list of a query tile.  Blocks [n_qt, n_qt + n_kt): query-tile list
-// of a key tile (backward only).  Order inside a list is ascending tile index.
-__global__ void k0_lists(Plan p, int for_bwd)
+// One block per query tile: its non-skipped key tiles, ascending.
+__global__ void k0_lists(Plan p)
 {
     __shared__ int warp_cnt[4];
     __shared__ int base;
-    const bool is_q = (int)blockIdx.x < p.n_qt;
-    if (!is_q && !for_bwd)
-        return;
-    const int self = is_q ? blockIdx.x : blockIdx.x - p.n_qt;
-    const int n_other = is_q ? p.n_kt : p.n_qt;
+    const int self = blockIdx.x;
     if (threadIdx.x == 0)
         base = 0;
     __syncthreads();
-    for (int o0 = 0; o0 < n_other; o0 += blockDim.x) {
+    for (int o0 = 0; o0 < p.n_kt; o0 += blockDim.x) {
         const int o = o0 + threadIdx.x;
         uint8_t c = TILE_SKIP;
-        if (o < n_other)
-            c = is_q ? p.cls[(size_t)self * p.n_kt + o] : p.cls[(size_t)o * p.n_kt + self];
+        if (o < p.n_kt)
+            c = p.cls[(size_t)self * p.n_kt + o];
         const unsigned bal = __ballot_sync(0xffffffffu, c != TILE_SKIP);
         const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
         if (lane == 0)
@@ -191,28 +186,20 @@ __global__ void k0_lists(Plan p, int for_bwd)
             off += warp_cnt[w];
         off += __popc(bal & ((1u << lane) - 1u));
         if (c != TILE_SKIP) {
-            if (is_q) {
-                const int2 kt = p.ktile[o];
-                p.klist[(size_t)self * p.n_kt + off] = make_int2(kt.x, kt.y | ((int)c << 16));
-            } else {
-                p.qlist[(size_t)self * p.n_qt + off] = make_int2(o, (int)c);
-            }
+            const int2 kt = p.ktile[o];
+            p.klist[(size_t)self * p.n_kt + off] = make_int2(kt.x, kt.y | ((int)c << 16));
         }
         __syncthreads();
         if (threadIdx.x == 0)
             base += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
         __syncthreads();
     }
-    if (threadIdx.x == 0) {
-        if (is_q)
-            p.kcount[self] = base;
-        else
-            p.qcount[self] = base;
-    }
+    if (threadIdx.x == 0)
+        p.kcount[self] = base;
 }
 
-// ---- 4b. order query tiles longest-first; cut the backward into work items ------------------
-__global__ void k0_schedule(Plan p, int for_bwd)
+// ---- 4b. order query tiles longest-first ----------------------------------------------------
+__global__ void k0_schedule(Plan p)
 {
     extern __shared__ int cnt[];
     const int n = p.n_qt;
@@ -231,50 +218,88 @@ __global__ void k0_schedule(Plan p, int for_bwd)
         for (int i = threadIdx.x; i < n; i += blockDim.x)
             p.qorder[i] = n - 1 - i;
     }
-    if (!for_bwd)
-        return;
-    // Work item = one key tile and up to BWD_CQ consecutive entries of its query-tile list.
-    // Key tiles with long lists come first because their items are all full-sized.
-    __shared__ int sum_big[1024], sum_small[1024];
-    __shared__ int total_big;
-    const int per = (p.n_kt + (int)blockDim.x - 1) / (int)blockDim.x;
-    const int k0 = min(p.n_kt, (int)threadIdx.x * per), k1 = min(p.n_kt, k0 + per);
-    int nb = 0, ns = 0;
-    for (int kt = k0; kt < k1; ++kt) {
-        const int c = p.qcount[kt];
-        const int chunks = (c + BWD_CQ - 1) / BWD_CQ;
-        if (c >= BWD_CQ)
-            nb += chunks;
-        else
-            ns += chunks;
-    }
-    sum_big[threadIdx.x] = nb;
-    sum_small[threadIdx.x] = ns;
+}
+
+// ---- 4c. backward work items ------------------------------------------------------------------
+// A backward work item is one key tile together with the non-skipped query tiles of one aligned
+// group of BWD_CQ consecutive query tiles ("chunk").  Items are laid out chunk-major so that the
+// CTAs running at the same time work on the same few query tiles: their Q / dO rows and their
+// fp32 dQ staging rows then stay in L2.
+// Pass 1, one block per chunk: for every key tile a 16-bit word (bit b: query tile 8c+b is not
+// skipped, bit 8+b: it is FULL), and the number of key tiles with a non-zero word.
+__global__ void k0_chunk_masks(Plan p)
+{
+    __shared__ int total;
+    const int c = blockIdx.x;
+    if (threadIdx.x == 0)
+        total = 0;
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int ab = 0, as = 0;
-        for (int i = 0; i < (int)blockDim.x; ++i) {
-            const int b = sum_big[i], sm = sum_small[i];
-            sum_big[i] = ab;
-            sum_small[i] = as;
-            ab += b;
-            as += sm;
+    int mine = 0;
+    for (int kt = threadIdx.x; kt < p.n_kt; kt += blockDim.x) {
+        unsigned m = 0;
+        for (int b = 0; b < BWD_CQ; ++b) {
+            const int qt = c * BWD_CQ + b;
+            if (qt < p.n_qt) {
+                const uint8_t cl = p.cls[(size_t)qt * p.n_kt + kt];
+                if (cl != TILE_SKIP)
+                    m |= 1u << b;
+                if (cl == TILE_FULL)
+                    m |= 1u << (8 + b);
+            }
         }
-        total_big = ab;
-        p.counters[1] = ab + as;
+        p.cmask[(size_t)c * p.n_kt + kt] = (uint16_t)m;
+        mine += (m != 0);
     }
+    for (int o = 16; o > 0; o >>= 1)
+        mine += __shfl_xor_sync(0xffffffffu, mine, o);
+    if ((threadIdx.x & 31) == 0)
+        atomicAdd(&total, mine);
     __syncthreads();
-    int ob = sum_big[threadIdx.x], os = total_big + sum_small[threadIdx.x];
-    for (int kt = k0; kt < k1; ++kt) {
-        const int c = p.qcount[kt];
-        for (int j = 0; j < c; j += BWD_CQ) {
-            const int4 item = make_int4(kt, j, min(BWD_CQ, c - j), 0);
-            if (c >= BWD_CQ)
-                p.bitems[ob++] = item;
-            else
-                p.bitems[os++] = item;
-        }
+    if (threadIdx.x == 0)
+        p.ccount[c] = total;
+}
+
+// Pass 2, one block per chunk: items of the chunk, key tiles ascending, behind the items of all
+// earlier chunks.  item = (key tile, chunk, mask word, query tiles in the item).
+__global__ void k0_chunk_items(Plan p)
+{
+    __shared__ int warp_cnt[4];
+    __shared__ int base;
+    const int c = blockIdx.x;
+    int before = 0;
+    for (int i = threadIdx.x; i < c; i += blockDim.x)
+        before += p.ccount[i];
+    for (int o = 16; o > 0; o >>= 1)
+        before += __shfl_xor_sync(0xffffffffu, before, o);
+    if (threadIdx.x == 0)
+        base = 0;
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0)
+        atomicAdd(&base, before);
+    __syncthreads();
+    for (int o0 = 0; o0 < p.n_kt; o0 += blockDim.x) {
+        const int kt = o0 + threadIdx.x;
+        unsigned m = 0;
+        if (kt < p.n_kt)
+            m = p.cmask[(size_t)c * p.n_kt + kt];
+        const unsigned bal = __ballot_sync(0xffffffffu, m != 0);
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+        if (lane == 0)
+            warp_cnt[wid] = __popc(bal);
+        __syncthreads();
+        int off = base;
+        for (int w = 0; w < wid; ++w)
+            off += warp_cnt[w];
+        off += __popc(bal & ((1u << lane) - 1u));
+        if (m != 0)
+            p.bitems[off] = make_int4(kt, c, (int)m, __popc(m & 0xffu));
+        __syncthreads();
+        if (threadIdx.x == 0)
+            base += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
+        __syncthreads();
     }
+    if (c == (int)gridDim.x - 1 && threadIdx.x == 0)
+        p.counters[1] = base;
 }
 
 // ---- test hook: the mask as the device predicate sees it -----------------------------------
@@ -318,10 +343,15 @@ int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int 
     k0_summaries<<<p.n_qt + p.n_kt, 128, 0, s>>>(p);
     k0_classify_quick<<<dim3((p.n_kt + 127) / 128, p.n_qt), 128, 0, s>>>(p);
     k0_classify_exact<<<592, 128, 0, s>>>(p);
-    k0_lists<<<p.n_qt + (for_bwd ? p.n_kt : 0), 128, 0, s>>>(p, for_bwd ? 1 : 0);
+    k0_lists<<<p.n_qt, 128, 0, s>>>(p);
     const int smem = (p.n_qt <= 8192 ? p.n_qt : 0) * (int)sizeof(int);
-    k0_schedule<<<1, 1024, smem, s>>>(p, for_bwd ? 1 : 0);
-    return 6;
+    k0_schedule<<<1, 1024, smem, s>>>(p);
+    if (!for_bwd)
+        return 6;
+    const int n_ch = (p.n_qt + BWD_CQ - 1) / BWD_CQ;
+    k0_chunk_masks<<<n_ch, 128, 0, s>>>(p);
+    k0_chunk_items<<<n_ch, 128, 0, s>>>(p);
+    return 8;
 }
 
 int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s)
