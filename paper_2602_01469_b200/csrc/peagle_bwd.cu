@@ -442,8 +442,11 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 //   while the compute warps turn S^T(i) into P^T(i):   dK(i-1), dQ(i-1), dP^T(i)
 //   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
 // and dQ(i-1) is drained to the fp32 staging rows after dS^T(i) has been handed over.  K / V of
-// the next work item are prefetched into a second stage.  384 threads: warps 0-7 compute, warp 8
-// issues MMAs, warp 9 produces, warps 10-11 only give their registers to the compute warps.
+// the next work item are prefetched into a second stage.  512 threads: warps 0-7 compute, warp 8
+// issues MMAs, warp 9 produces, warps 12-15 drain dQ (and dK / dV at the end of a work item) from
+// tensor memory to the fp32 buffers with global reductions.  The drain has warps of its own
+// because a thread with reductions in flight stalls on its next proxy fence, which the compute
+// warps need once per step for the dS^T hand-over.
 struct Bwd64Cfg {
     static constexpr int D = 64;
     static constexpr int NSQ = 3;
@@ -511,7 +514,7 @@ struct BwdWalk {
     }
 };
 
-__global__ void __launch_bounds__(384, 1)
+__global__ void __launch_bounds__(512, 1)
 bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
              const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
              const BwdParams P)
@@ -536,20 +539,20 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < NSQ; ++s) {
-            mbar_init(BAR(B_QFULL + s), 1);
+            mbar_init(BAR(B_QFULL + s), 2); // the TMA transaction + the row buffer
             mbar_init(BAR(B_QEMPTY + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
             mbar_init(BAR(B_KVFULL + s), 1);
             mbar_init(BAR(B_KVEMPTY + s), 1);
             mbar_init(BAR(B_DQFULL + s), 1);
-            mbar_init(BAR(B_DQEMPTY + s), 256);
+            mbar_init(BAR(B_DQEMPTY + s), 128);
         }
         mbar_init(BAR(B_SFULL), 1);
         mbar_init(BAR(B_DPFULL), 1);
         mbar_init(BAR(B_PFULL), 256);
         mbar_init(BAR(B_DSFULL), 256);
-        mbar_init(BAR(B_ACCFREE), 256);
+        mbar_init(BAR(B_ACCFREE), 128);
         fence_mbar_init();
     }
     if (warp == 8) {
@@ -561,7 +564,81 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp >= 8) {
+    if (warp >= 12) {
+        // ------------------------------------------------------------ drain (warps 12-15)
+        reg_dec<104>();
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const int sub = lane >> 2, cq = 2 * (lane & 3); // row inside a 16-lane load, first column
+        BwdWalk wk;
+        wk.init(P, blockIdx.x, gridDim.x);
+        int2 ktile = make_int2(0, 0);
+        bool ok = true;
+        // adds a [32 lanes x 64 columns] block of tensor memory, scaled, to fp32 rows in global
+        // memory: row_of(lane) gives the destination row pointer or null
+        auto drain_block = [&](uint32_t tcol, float f, auto row_ptr, int barrier) {
+            uint32_t o[2][32];
+            tmem_ld_16x256b_x8(tmem + lane_base + tcol, o[0]);
+            tmem_ld_16x256b_x8(tmem + lane_base + (16u << 16) + tcol, o[1]);
+            tmem_wait_ld();
+            if (barrier >= 0) {
+                tc_fence_before();
+                mbar_arrive(BAR(barrier));
+            }
+#pragma unroll
+            for (int hf = 0; hf < 2; ++hf) {
+                float *ra = row_ptr((warp & 3) * 32 + hf * 16 + sub);
+                float *rb = row_ptr((warp & 3) * 32 + hf * 16 + sub + 8);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    if (ra)
+                        red_add_v2(ra + 8 * i + cq, __uint_as_float(o[hf][4 * i]) * f,
+                                   __uint_as_float(o[hf][4 * i + 1]) * f);
+                    if (rb)
+                        red_add_v2(rb + 8 * i + cq, __uint_as_float(o[hf][4 * i + 2]) * f,
+                                   __uint_as_float(o[hf][4 * i + 3]) * f);
+                }
+            }
+        };
+        for (int it = 0; ok && wk.valid; ++it) {
+            if (wk.first())
+                ktile = P.ktile[wk.kt];
+            const int row0 = P.q_begin + wk.qt() * BM;
+            const int h = wk.head();
+            const bool last = wk.last();
+            ok = __all_sync(0xffffffffu,
+                            mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag));
+            if (!ok)
+                break;
+            tc_fence_after();
+            drain_block(C::TM_DQ + (it & 1) * 64, P.scale,
+                        [&](int i) -> float * {
+                            const int row = row0 + i;
+                            return row < P.q_end
+                                       ? P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D
+                                       : nullptr;
+                        },
+                        B_DQEMPTY + (it & 1));
+            if (last) {
+                // every MMA of the work item is complete (the barrier above covers them all)
+                const int g = wk.g;
+                drain_block(C::TM_DK, P.scale,
+                            [&](int i) -> float * {
+                                return i < ktile.y
+                                           ? P.dK_acc + ((size_t)(ktile.x + i) * P.Hkv + g) * D
+                                           : nullptr;
+                            },
+                            -1);
+                drain_block(C::TM_DV, 1.f,
+                            [&](int i) -> float * {
+                                return i < ktile.y
+                                           ? P.dV_acc + ((size_t)(ktile.x + i) * P.Hkv + g) * D
+                                           : nullptr;
+                            },
+                            B_ACCFREE);
+            }
+            wk.next();
+        }
+    } else if (warp >= 8) {
         reg_dec<56>();
         if (warp == 9) {
             // -------------------------------------------------------- producer
@@ -597,6 +674,12 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
                 if (!ok)
                     break;
+                if (lane == 0) {
+                    mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * TB);
+                    const uint32_t qa = sb + C::OFF_Q + st * 2 * TB;
+                    tma_load_3d(qa, &tmQ, BAR(B_QFULL + st), 0, h, row0);
+                    tma_load_3d(qa + TB, &tmdO, BAR(B_QFULL + st), 0, h, row0);
+                }
                 float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
                 for (int i = lane; i < BM; i += 32) {
                     const int row = row0 + i;
@@ -616,12 +699,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     reinterpret_cast<int *>(rowbuf)[256 + i] = mq;
                 }
                 __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * TB);
-                    const uint32_t qa = sb + C::OFF_Q + st * 2 * TB;
-                    tma_load_3d(qa, &tmQ, BAR(B_QFULL + st), 0, h, row0);
-                    tma_load_3d(qa + TB, &tmdO, BAR(B_QFULL + st), 0, h, row0);
-                }
+                if (lane == 0)
+                    mbar_arrive(BAR(B_QFULL + st));
                 const bool was_last = wk.last();
                 wk.next();
                 if (was_last && wk.valid)
@@ -632,18 +711,25 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
             constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
             constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
-            const uint32_t dsa = sb + C::OFF_DS;
-            auto issue_s = [&](uint32_t ka, uint32_t qa) {
+            // Lower descriptor words (16-byte units).  "k" = K-major operand, "m" = MN-major.
+            const uint32_t ds_k = desc_lo_sw128(sb + C::OFF_DS, 16);
+            const uint32_t ds_m = desc_lo_sw128(sb + C::OFF_DS, TB);
+            const uint32_t kv_k = desc_lo_sw128(sb + C::OFF_KV, 16);
+            const uint32_t kv_m = desc_lo_sw128(sb + C::OFF_KV, TB);
+            const uint32_t q_k = desc_lo_sw128(sb + C::OFF_Q, 16);
+            const uint32_t q_m = desc_lo_sw128(sb + C::OFF_Q, TB);
+            constexpr uint32_t TBU = TB >> 4; // one tile in descriptor units
+            // S^T = K Q^T and dP^T = V dO^T: kv / q are the stage offsets in descriptor units
+            auto issue_s = [&](uint32_t kv, uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem + C::TM_S, smem_desc_sw128(ka + k * 32, 16, 1024),
-                           smem_desc_sw128(qa + k * 32, 16, 1024), IDESC_S, k > 0);
+                    mma_ss_lo(tmem + C::TM_S, kv_k + kv + k * 2, q_k + q + k * 2, IDESC_S, k > 0);
             };
-            auto issue_dp = [&](uint32_t va, uint32_t doa) {
+            auto issue_dp = [&](uint32_t kv, uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss(tmem + C::TM_DP, smem_desc_sw128(va + k * 32, 16, 1024),
-                           smem_desc_sw128(doa + k * 32, 16, 1024), IDESC_S, k > 0);
+                    mma_ss_lo(tmem + C::TM_DP, kv_k + kv + TBU + k * 2, q_k + q + TBU + k * 2, IDESC_S,
+                              k > 0);
             };
             BwdWalk cur, nxt;
             cur.init(P, blockIdx.x, gridDim.x);
@@ -656,23 +742,20 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                      mbar_wait(BAR(B_QFULL + 0), 0, abort_flag);
                 if (ok) {
                     tc_fence_after();
-                    const uint32_t ka = sb + C::OFF_KV, qa = sb + C::OFF_Q;
-                    issue_s(ka, qa);
+                    issue_s(0, 0);
                     tc_commit(BAR(B_SFULL));
-                    issue_dp(ka + TB, qa + TB);
+                    issue_dp(0, 0);
                     tc_commit(BAR(B_DPFULL));
                 }
             }
             for (int it = 0; ok && cur.valid; ++it) {
                 const int st = it % NSQ;
                 const int ks = cur.w & 1;
-                const uint32_t ka = sb + C::OFF_KV + 2 * ks * TB;
-                const uint32_t qa = sb + C::OFF_Q + st * 2 * TB, doa = qa + TB;
+                const uint32_t kvo = 2 * ks * TBU, qo = st * 2 * TBU;
                 const bool first = cur.first(), last = cur.last();
                 const int nst = (it + 1) % NSQ, nph = ((it + 1) / NSQ) & 1;
                 const int nks = nxt.valid ? (nxt.w & 1) : 0;
-                const uint32_t nka = sb + C::OFF_KV + 2 * nks * TB;
-                const uint32_t nqa = sb + C::OFF_Q + nst * 2 * TB;
+                const uint32_t nkvo = 2 * nks * TBU, nqo = nst * 2 * TBU;
                 // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
                 ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
                 if (ok && first)
@@ -682,8 +765,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    mma_ts(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
-                           smem_desc_sw128(doa + k * 2048, TB, 1024), IDESC_KV, !first || k > 0);
+                    mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                              q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
                 if (nxt.valid) {
                     if (nxt.first())
                         ok = mbar_wait(BAR(B_KVFULL + nks), (nxt.w >> 1) & 1, abort_flag);
@@ -691,7 +774,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     if (!ok)
                         break;
                     tc_fence_after();
-                    issue_s(nka, nqa);
+                    issue_s(nkvo, nqo);
                     tc_commit(BAR(B_SFULL));
                 }
                 // ---- dK(it), dQ(it) once dS^T(it) is in shared memory, then dP^T(it+1)
@@ -702,18 +785,18 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    mma_ss(tmem + C::TM_DK, smem_desc_sw128(dsa + (k / 4) * TB + (k % 4) * 32, 16, 1024),
-                           smem_desc_sw128(qa + k * 2048, TB, 1024), IDESC_KV, !first || k > 0);
+                    mma_ss_lo(tmem + C::TM_DK, ds_k + (k / 4) * TBU + (k % 4) * 2, q_m + qo + k * 128,
+                              IDESC_KV, !first || k > 0);
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    mma_ss(tmem + C::TM_DQ + (it & 1) * 64, smem_desc_sw128(dsa + k * 2048, TB, 1024),
-                           smem_desc_sw128(ka + k * 2048, TB, 1024), IDESC_DQ, k > 0);
+                    mma_ss_lo(tmem + C::TM_DQ + (it & 1) * 64, ds_m + k * 128, kv_m + kvo + k * 128,
+                              IDESC_DQ, k > 0);
                 tc_commit(BAR(B_DQFULL + (it & 1)));
                 tc_commit(BAR(B_QEMPTY + st));
                 if (last)
                     tc_commit(BAR(B_KVEMPTY + ks));
                 if (nxt.valid) {
-                    issue_dp(nka + TB, nqa + TB);
+                    issue_dp(nkvo, nqo);
                     tc_commit(BAR(B_DPFULL));
                 }
                 cur = nxt;
@@ -722,50 +805,25 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
         }
     } else {
-        reg_inc<224>();
+        reg_inc<176>();
         // ------------------------------------------------------------ compute (warps 0-7)
         const int wg = warp >> 2;
         const int r = threadIdx.x & 127; // key lane for S/dP/dK/dV, query row for dQ
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_sel + C::TM_S + wg * 64;
         const uint32_t tDP = tmem + lane_sel + C::TM_DP + wg * 64;
-        const uint32_t tDQ = tmem + lane_sel + C::TM_DQ + wg * 32;
-        const uint32_t tACC = tmem + lane_sel + (wg == 0 ? C::TM_DK : C::TM_DV);
         uint8_t *dsrow = sp + C::OFF_DS + wg * TB + r * 128;
         BwdWalk wk;
         wk.init(P, blockIdx.x, gridDim.x);
         bool ok = true;
-        bool pending = false;   // dQ of the previous iteration still sits in tensor memory
-        int prev_row0 = 0, prev_h = 0;
         int32_t mk = META_NONE_K;
-        int2 ktile = make_int2(0, 0);
-        // dQ(j) -> fp32 staging rows; j's accumulator is TM_DQ + (j & 1) * 64
-        auto drain_dq = [&](int j, int row0, int h) {
-            const int row = row0 + r;
-            float *dst = P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D + wg * 32;
-            uint32_t o[32];
-            tmem_ld32(tDQ + (j & 1) * 64, o);
-            tmem_wait_ld();
-            if (row < P.q_end) {
-#pragma unroll
-                for (int i = 0; i < 32; i += 4)
-                    red_add_v4(dst + i, __uint_as_float(o[i]) * P.scale,
-                               __uint_as_float(o[i + 1]) * P.scale,
-                               __uint_as_float(o[i + 2]) * P.scale,
-                               __uint_as_float(o[i + 3]) * P.scale);
-            }
-            tc_fence_before();
-            mbar_arrive(BAR(B_DQEMPTY + (j & 1)));
-        };
         for (int it = 0; ok && wk.valid; ++it) {
             const int st = it % NSQ, ph = (it / NSQ) & 1;
             if (wk.first()) {
-                ktile = P.ktile[wk.kt];
+                const int2 ktile = P.ktile[wk.kt];
                 mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
             }
-            const int row0 = P.q_begin + wk.qt() * BM;
-            const int h = wk.head();
-            const bool full = wk.full(), last = wk.last();
+            const bool full = wk.full();
             const float *rowbuf = reinterpret_cast<const float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
             const float4 *nl4 = reinterpret_cast<const float4 *>(rowbuf + wg * 64);
             const float4 *nd4 = reinterpret_cast<const float4 *>(rowbuf + 128 + wg * 64);
@@ -854,42 +912,6 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = dsv[j];
             fence_proxy_async_smem();
             mbar_arrive(BAR(B_DSFULL));
-            // ---- dQ of the previous iteration (its MMAs are done: waited on above)
-            if (pending) {
-                tc_fence_after();
-                drain_dq(it - 1, prev_row0, prev_h);
-                pending = false;
-            }
-            if (last) {
-                // end of the work item: dQ of this iteration, then dK (group 0) / dV (group 1)
-                ok = __all_sync(0xffffffffu,
-                                mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag));
-                if (!ok)
-                    break;
-                tc_fence_after();
-                drain_dq(it, row0, h);
-                float *acc = (wg == 0 ? P.dK_acc : P.dV_acc) + ((size_t)(ktile.x + r) * P.Hkv + wk.g) * D;
-                const float f = (wg == 0) ? P.scale : 1.f;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tACC + c * 32, o);
-                    tmem_wait_ld();
-                    if (r < ktile.y) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            red_add_v4(acc + c * 32 + i, __uint_as_float(o[i]) * f,
-                                       __uint_as_float(o[i + 1]) * f, __uint_as_float(o[i + 2]) * f,
-                                       __uint_as_float(o[i + 3]) * f);
-                    }
-                }
-                tc_fence_before();
-                mbar_arrive(BAR(B_ACCFREE));
-            } else {
-                pending = true;
-                prev_row0 = row0;
-                prev_h = h;
-            }
             wk.next();
         }
     }
@@ -1032,7 +1054,7 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         if (ev0)
             cudaEventRecord(ev0, s);
         if (D == 64)
-            bwd64_kernel<<<n_sm, 384, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+            bwd64_kernel<<<n_sm, 512, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
         else
             bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
         if (ev1)
