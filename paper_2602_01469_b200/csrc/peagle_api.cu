@@ -254,9 +254,10 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
         return PEAGLE_OK;
     const size_t q_len = (size_t)(c.plan.q_end - c.plan.q_begin);
     const size_t Hq = (size_t)prob->n_q_heads, D = (size_t)prob->head_dim;
-    const size_t delta_bytes = ((Hq * q_len * 4 + 255) / 256) * 256;
+    const size_t q_pad = (size_t)c.plan.n_qt * BM;
+    const size_t row_bytes = ((2 * Hq + 1) * q_pad * 4 + 255) / 256 * 256;
     const size_t dq_bytes = q_len * Hq * D * 4;
-    int rc = ensure(ctx, ctx->bwd_buf, delta_bytes + dq_bytes + 256, s);
+    int rc = ensure(ctx, ctx->bwd_buf, row_bytes + dq_bytes + 256, s);
     if (rc != PEAGLE_OK)
         return rc;
     BwdArgs a;
@@ -269,8 +270,10 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
     a.dQ = dQ;
     a.dK_acc = dK_acc;
     a.dV_acc = dV_acc;
-    a.delta = static_cast<float *>(ctx->bwd_buf.ptr);
-    a.dq_acc = reinterpret_cast<float *>(static_cast<uint8_t *>(ctx->bwd_buf.ptr) + delta_bytes);
+    a.nl2 = static_cast<float *>(ctx->bwd_buf.ptr);
+    a.nd = a.nl2 + Hq * q_pad;
+    a.mqp = reinterpret_cast<int32_t *>(a.nd + Hq * q_pad);
+    a.dq_acc = reinterpret_cast<float *>(static_cast<uint8_t *>(ctx->bwd_buf.ptr) + row_bytes);
     a.Hq = prob->n_q_heads;
     a.Hkv = prob->n_kv_heads;
     a.D = prob->head_dim;

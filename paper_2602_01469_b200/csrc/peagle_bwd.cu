@@ -33,9 +33,10 @@ struct BwdParams {
     const int32_t *meta;
     int *status;
     int n_qt, q_begin, q_end, T;
-    const float *LSE;
-    const float *delta; // [Hq][q_len]
-    float *dq_acc;      // [q_len][Hq][D]
+    const float *nl2, *nd; // [Hq][q_pad] -LSE*log2(e) and -Delta, padded rows (-inf, 0)
+    const int32_t *mqp;    // [q_pad] packed metadata of the partition's rows
+    int q_pad;             // n_qt * BM
+    float *dq_acc;         // [q_len][Hq][D]
     float *dK_acc, *dV_acc;
     int Hq, Hkv;
     float scale, scale_log2;
@@ -162,20 +163,10 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
                     for (int i = lane; i < BM; i += 32) {
                         const int row = row0 + i;
-                        float l2 = CUDART_INF_F, dl = 0.f;
-                        int mq = META_NONE_Q;
-                        if (row < P.q_end) {
-                            const float lse = P.LSE[(size_t)h * P.T + row];
-                            if (lse != -CUDART_INF_F)
-                                l2 = lse * 1.4426950408889634f;
-                            dl = P.delta[(size_t)h * (P.q_end - P.q_begin) + (row - P.q_begin)];
-                            mq = P.meta[row];
-                            if (mq == META_NONE_K)
-                                mq = META_NONE_Q;
-                        }
-                        rowbuf[i] = l2;
-                        rowbuf[128 + i] = dl;
-                        reinterpret_cast<int *>(rowbuf)[256 + i] = mq;
+                        const size_t ri = (size_t)h * P.q_pad + (row - P.q_begin);
+                        rowbuf[i] = -P.nl2[ri];
+                        rowbuf[128 + i] = -P.nd[ri];
+                        reinterpret_cast<int *>(rowbuf)[256 + i] = P.mqp[row - P.q_begin];
                     }
                     __syncwarp();
                     if (lane == 0) {
@@ -539,7 +530,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         for (int s = 0; s < NSQ; ++s) {
-            mbar_init(BAR(B_QFULL + s), 2); // the TMA transaction + the row buffer
+            mbar_init(BAR(B_QFULL + s), 1);
             mbar_init(BAR(B_QEMPTY + s), 1);
         }
         for (int s = 0; s < 2; ++s) {
@@ -675,32 +666,16 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (!ok)
                     break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * TB);
+                    mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * TB + C::ROW_BYTES);
                     const uint32_t qa = sb + C::OFF_Q + st * 2 * TB;
                     tma_load_3d(qa, &tmQ, BAR(B_QFULL + st), 0, h, row0);
                     tma_load_3d(qa + TB, &tmdO, BAR(B_QFULL + st), 0, h, row0);
+                    const uint32_t ra = sb + C::OFF_ROW + st * C::ROW_BYTES;
+                    const size_t ri = (size_t)h * P.q_pad + (size_t)wk.qt() * BM;
+                    bulk_load(ra, P.nl2 + ri, 512, BAR(B_QFULL + st));
+                    bulk_load(ra + 512, P.nd + ri, 512, BAR(B_QFULL + st));
+                    bulk_load(ra + 1024, P.mqp + (size_t)wk.qt() * BM, 512, BAR(B_QFULL + st));
                 }
-                float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
-                for (int i = lane; i < BM; i += 32) {
-                    const int row = row0 + i;
-                    float nl2 = -CUDART_INF_F, ndl = 0.f;
-                    int mq = META_NONE_Q;
-                    if (row < P.q_end) {
-                        const float lse = P.LSE[(size_t)h * P.T + row];
-                        if (lse != -CUDART_INF_F)
-                            nl2 = -lse * 1.4426950408889634f;
-                        ndl = -P.delta[(size_t)h * (P.q_end - P.q_begin) + (row - P.q_begin)];
-                        mq = P.meta[row];
-                        if (mq == META_NONE_K)
-                            mq = META_NONE_Q;
-                    }
-                    rowbuf[i] = nl2;
-                    rowbuf[128 + i] = ndl;
-                    reinterpret_cast<int *>(rowbuf)[256 + i] = mq;
-                }
-                __syncwarp();
-                if (lane == 0)
-                    mbar_arrive(BAR(B_QFULL + st));
                 const bool was_last = wk.last();
                 wk.next();
                 if (was_last && wk.valid)
@@ -934,17 +909,24 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     }
 }
 
-// Delta[h][r] = <dO[q,h,:], O[q,h,:]> for the rows of the partition, and zero the fp32 dQ staging.
+// Per-row inputs of the backward kernels for the q_pad = n_qt * BM rows the query tiles cover:
+// -LSE * log2(e), -Delta with Delta[h][r] = <dO[q,h,:], O[q,h,:]>, and the packed metadata, with
+// neutral values for the rows past the partition's end.  Also zeroes the fp32 dQ staging.
 template <int D>
 __global__ void bwd_prepare(const __nv_bfloat16 *__restrict__ O, const __nv_bfloat16 *__restrict__ dO,
-                            float *__restrict__ delta, float *__restrict__ dq_acc, int q_begin,
-                            int q_len, int Hq)
+                            const float *__restrict__ LSE, const int32_t *__restrict__ meta,
+                            float *__restrict__ nl2, float *__restrict__ nd,
+                            int32_t *__restrict__ mqp, float *__restrict__ dq_acc, int q_begin,
+                            int q_len, int q_pad, int Hq, int T)
 {
     constexpr int TPR = D / 8; // threads per (row, head)
     const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const size_t n = (size_t)q_len * Hq * TPR;
+    const size_t n = (size_t)q_pad * Hq * TPR;
+    const size_t rh = gid / TPR;
+    const size_t r = rh / Hq, h = rh % Hq;
+    const bool real = gid < n && r < (size_t)q_len;
     float acc = 0.f;
-    if (gid < n) {
+    if (real) {
         const size_t src = (size_t)q_begin * Hq * D + gid * 8;
         const uint4 a = *reinterpret_cast<const uint4 *>(O + src);
         const uint4 b = *reinterpret_cast<const uint4 *>(dO + src);
@@ -963,9 +945,20 @@ __global__ void bwd_prepare(const __nv_bfloat16 *__restrict__ O, const __nv_bflo
     for (int o = TPR / 2; o > 0; o >>= 1)
         acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (gid < n && (gid % TPR) == 0) {
-        const size_t rh = gid / TPR;
-        const size_t r = rh / Hq, h = rh % Hq;
-        delta[h * (size_t)q_len + r] = acc;
+        float l = -CUDART_INF_F;
+        int mq = META_NONE_Q;
+        if (real) {
+            const float lse = LSE[h * (size_t)T + q_begin + r];
+            if (lse != -CUDART_INF_F)
+                l = -lse * 1.4426950408889634f;
+            mq = meta[q_begin + r];
+            if (mq == META_NONE_K)
+                mq = META_NONE_Q;
+        }
+        nl2[h * (size_t)q_pad + r] = l;
+        nd[h * (size_t)q_pad + r] = real ? -acc : 0.f;
+        if (h == 0)
+            mqp[r] = mq;
     }
 }
 
@@ -1015,10 +1008,12 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         make_bf16_map(enc, &tmK, a.K, D, a.Hkv, p.T) || make_bf16_map(enc, &tmV, a.V, D, a.Hkv, p.T))
         return PEAGLE_ERR_CUDA;
     const int q_len = p.q_end - p.q_begin;
+    const int q_pad = p.n_qt * BM;
     const size_t n_prep = (size_t)q_len * a.Hq * (D / 8);
-    bwd_prepare<D><<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
-        static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.delta,
-        a.dq_acc, p.q_begin, q_len, a.Hq);
+    const size_t n_prep_pad = (size_t)q_pad * a.Hq * (D / 8);
+    bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
+        static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.LSE,
+        p.meta, a.nl2, a.nd, a.mqp, a.dq_acc, p.q_begin, q_len, q_pad, a.Hq, p.T);
     int launches = 1;
     if (p.n_kt > 0) {
         BwdParams P;
@@ -1031,8 +1026,10 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         P.q_begin = p.q_begin;
         P.q_end = p.q_end;
         P.T = p.T;
-        P.LSE = a.LSE;
-        P.delta = a.delta;
+        P.nl2 = a.nl2;
+        P.nd = a.nd;
+        P.mqp = a.mqp;
+        P.q_pad = q_pad;
         P.dq_acc = a.dq_acc;
         P.dK_acc = a.dK_acc;
         P.dV_acc = a.dV_acc;

@@ -59,7 +59,10 @@ struct BwdArgs {
     const float *LSE;
     void *dQ;
     float *dK_acc, *dV_acc;
-    float *delta;   // [Hq][q_len] scratch
+    // per-row scratch of the call, q_pad = query tiles * BM rows, rows past the partition padded
+    float *nl2;     // [Hq][q_pad] -LSE * log2(e); -inf for a padded row or a row that saw no key
+    float *nd;      // [Hq][q_pad] -Delta = -<dO, O>; 0 for a padded row
+    int32_t *mqp;   // [q_pad] packed metadata of the partition's rows; META_NONE_Q when padded
     float *dq_acc;  // [q_len][Hq][D] scratch, fp32
     int Hq, Hkv, D;
     float scale;

@@ -95,6 +95,15 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap *m, 
         "l"(reinterpret_cast<uint64_t>(m)), "r"(bar), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// Untiled bulk copy global -> shared (both 16-byte aligned, size % 16 == 0); completes `bytes`
+// on the mbarrier.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar)
+        : "memory");
+}
 // Bulk reduce-add of fp32 from shared to global memory (both 16-byte aligned, size % 16 == 0).
 __device__ __forceinline__ void bulk_reduce_add_f32(void *gdst, uint32_t ssrc, uint32_t bytes)
 {
