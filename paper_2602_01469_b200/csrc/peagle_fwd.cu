@@ -56,7 +56,7 @@ struct FwdCfg {
 };
 
 template <int D>
-__global__ void __launch_bounds__(320, 1)
+__global__ void __launch_bounds__(384, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const FwdParams P)
 {
@@ -113,7 +113,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 9) {
+    // Warps 8-11 hand most of their registers to the eight softmax warps.
+    if (warp >= 8)
+        reg_dec<56>();
+    if (warp >= 10) {
+    } else if (warp == 9) {
         // ------------------------------------------------------------ producer
         if (cnt > 0) {
             if (lane == 0) {
@@ -159,23 +163,24 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         if (lane == 0 && cnt > 0) {
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, BN, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16_f32(128, D, 0, 1);
+            // lower descriptor words in 16-byte units (see desc_lo_sw128)
+            const uint32_t q_lo = desc_lo_sw128(sb + C::OFF_Q, 16);
+            const uint32_t k_lo = desc_lo_sw128(sb + C::OFF_K, 16);
+            const uint32_t v_lo = desc_lo_sw128(sb + C::OFF_V, C::PANEL_BYTES);
+            constexpr uint32_t TU = C::TILE_BYTES >> 4, PU = C::PANEL_BYTES >> 4;
             auto issue_s = [&](int x, int st) {
-                const uint32_t qa = sb + C::OFF_Q + x * C::TILE_BYTES;
-                const uint32_t ka = sb + C::OFF_K + st * C::TILE_BYTES;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
-                    const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
-                    mma_ss(tmem + C::TM_S + x * 128, smem_desc_sw128(qa + off, 16, 1024),
-                           smem_desc_sw128(ka + off, 16, 1024), IDESC_S, k > 0);
+                    const uint32_t off = (k / 4) * PU + (k % 4) * 2;
+                    mma_ss_lo(tmem + C::TM_S + x * 128, q_lo + x * TU + off, k_lo + st * TU + off,
+                              IDESC_S, k > 0);
                 }
             };
             auto issue_pv = [&](int x, int st, bool acc) {
-                const uint32_t va = sb + C::OFF_V + st * C::TILE_BYTES;
 #pragma unroll
                 for (int k = 0; k < BN / 16; ++k)
-                    mma_ts(tmem + C::TM_O + x * D, tmem + C::TM_S + x * 128 + k * 8,
-                           smem_desc_sw128(va + k * 2048, C::PANEL_BYTES, 1024), IDESC_O,
-                           acc || k > 0);
+                    mma_ts_lo(tmem + C::TM_O + x * D, tmem + C::TM_S + x * 128 + k * 8,
+                              v_lo + st * TU + k * 128, IDESC_O, acc || k > 0);
             };
             bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag) &&
                       mbar_wait(BAR(B_KFULL + 0), 0, abort_flag);
@@ -214,6 +219,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
     } else if (warp < 4 * ntile) {
+        reg_inc<224>();
         // ------------------------------------------------------------ softmax of tile x
         const int x = warp >> 2;
         const int r = threadIdx.x & 127;
@@ -416,7 +422,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     const int n_hb = P.two ? a.Hq / 2 : a.Hq;
     if (ev0)
         cudaEventRecord(ev0, s);
-    fwd_kernel<D><<<p.n_qt * n_hb, 320, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
+    fwd_kernel<D><<<p.n_qt * n_hb, 384, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
     if (ev1)
         cudaEventRecord(ev1, s);
     return 1;
