@@ -48,11 +48,17 @@ struct FwdCfg {
     static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
     static constexpr int OFF_META = OFF_V + NS * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_META + NS * BN * 4;
-    static constexpr int N_BAR = 1 + 4 * NS + 6;
+    static constexpr int N_BAR = 1 + 4 * NS + 8;
     static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024; // + slack for 1024-byte alignment
     static constexpr int TM_S = 0;      // S_A at 0, S_B at 128
     static constexpr int TM_O = 256;    // O_A at 256, O_B at 256 + D
+    // head_dim 64 leaves 128 columns for the bf16 probabilities (64 columns per tile), so the next
+    // S can be computed while the softmax of the current one runs.  head_dim 128 fills tensor
+    // memory with S and O, and P overwrites the first 64 columns of its own S.
+    static constexpr bool P_SEPARATE = (D == 64);
+    static constexpr int TM_P = P_SEPARATE ? 384 : 0;   // P_A, then P_B at + P_STRIDE
+    static constexpr int P_STRIDE = P_SEPARATE ? 64 : 128;
 };
 
 template <int D>
@@ -72,7 +78,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     // barrier indices
     constexpr int B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 1 + NS, B_VFULL = 1 + 2 * NS,
                   B_VEMPTY = 1 + 3 * NS, B_SFULL = 1 + 4 * NS, B_PFULL = B_SFULL + 2,
-                  B_ODONE = B_SFULL + 4;
+                  B_PVDONE = B_SFULL + 4, B_SREAD = B_SFULL + 6;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
     int32_t *smeta = reinterpret_cast<int32_t *>(sp + C::OFF_META);
@@ -93,14 +99,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         mbar_init(BAR(B_QFULL), 1);
         for (int s = 0; s < NS; ++s) {
             mbar_init(BAR(B_KFULL + s), 1);
-            mbar_init(BAR(B_KEMPTY + s), 1);
+            mbar_init(BAR(B_KEMPTY + s), P.two ? 2 : 1); // one commit per MMA-issuing thread
             mbar_init(BAR(B_VFULL + s), 1);
-            mbar_init(BAR(B_VEMPTY + s), 1);
+            mbar_init(BAR(B_VEMPTY + s), P.two ? 2 : 1);
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(BAR(B_SFULL + x), 1);
             mbar_init(BAR(B_PFULL + x), 128);
-            mbar_init(BAR(B_ODONE + x), 1);
+            mbar_init(BAR(B_PVDONE + x), 1);
+            mbar_init(BAR(B_SREAD + x), 128);
         }
         fence_mbar_init();
     }
@@ -116,8 +123,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     // Warps 8-11 hand most of their registers to the eight softmax warps.
     if (warp >= 8)
         reg_dec<56>();
-    if (warp >= 10) {
-    } else if (warp == 9) {
+    if (warp == 9) {
         // ------------------------------------------------------------ producer
         if (cnt > 0) {
             if (lane == 0) {
@@ -130,10 +136,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         tma_load_3d(sb + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmQ,
                                     BAR(B_QFULL), pn * 64, h0 + x, row0);
             }
+            // List entries and key metadata are fetched one key tile ahead, so that no global
+            // load latency sits between a stage becoming free and its TMA loads.
+            auto tile_meta = [&](int2 e, int32_t (&mv)[BN / 32]) {
+                const int start = e.x, len = e.y & 0xffff;
+                const bool need = (e.y >> 16) != TILE_FULL; // FULL tiles skip the predicate
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i) {
+                    const int t = lane + 32 * i;
+                    mv[i] = (need && t < len) ? P.meta[start + t] : META_NONE_K;
+                }
+            };
+            int2 e_cur = klist[0];
+            int2 e_nxt = cnt > 1 ? klist[1] : e_cur;
+            int32_t m_cur[BN / 32], m_nxt[BN / 32];
+            tile_meta(e_cur, m_cur);
             for (int j = 0; j < cnt; ++j) {
                 const int st = j % NS, ph = (j / NS) & 1;
-                const int2 e = klist[j];
-                const int start = e.x, len = e.y & 0xffff;
+                const int start = e_cur.x;
+                const int2 e_nn = j + 2 < cnt ? klist[j + 2] : e_nxt;
+                if (j + 1 < cnt)
+                    tile_meta(e_nxt, m_nxt);
                 bool ok = true;
                 if (lane == 0) {
                     ok = mbar_wait(BAR(B_KEMPTY + st), ph ^ 1, abort_flag);
@@ -147,8 +170,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 ok = ok && mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, abort_flag);
                 if (!__all_sync(0xffffffffu, ok))
                     break;
-                for (int i = lane; i < BN; i += 32)
-                    smeta[st * BN + i] = (i < len) ? P.meta[start + i] : META_NONE_K;
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i)
+                    smeta[st * BN + lane + 32 * i] = m_cur[i];
                 __syncwarp();
                 if (lane == 0) {
                     mbar_arrive_expect_tx(BAR(B_VFULL + st), C::TILE_BYTES);
@@ -156,64 +180,82 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         tma_load_3d(sb + C::OFF_V + st * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmV,
                                     BAR(B_VFULL + st), pn * 64, g, start);
                 }
+                e_cur = e_nxt;
+                e_nxt = e_nn;
+#pragma unroll
+                for (int i = 0; i < BN / 32; ++i)
+                    m_cur[i] = m_nxt[i];
             }
         }
-    } else if (warp == 8) {
+    } else if (warp == 8 || warp == 10) {
         // ------------------------------------------------------------ MMA issue
-        if (lane == 0 && cnt > 0) {
+        // Lane 0 of warp 8 issues every MMA of tile A, lane 0 of warp 10 those of tile B: the two
+        // tiles are independent instruction streams (they only share the K / V stages, which are
+        // released once both threads have committed), and two threads issue twice as fast as one.
+        const int x = (warp - 8) >> 1;
+        if (lane == 0 && cnt > 0 && x < ntile) {
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, BN, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16_f32(128, D, 0, 1);
+            constexpr uint32_t TU = C::TILE_BYTES >> 4, PU = C::PANEL_BYTES >> 4;
             // lower descriptor words in 16-byte units (see desc_lo_sw128)
-            const uint32_t q_lo = desc_lo_sw128(sb + C::OFF_Q, 16);
+            const uint32_t q_lo = desc_lo_sw128(sb + C::OFF_Q, 16) + x * TU;
             const uint32_t k_lo = desc_lo_sw128(sb + C::OFF_K, 16);
             const uint32_t v_lo = desc_lo_sw128(sb + C::OFF_V, C::PANEL_BYTES);
-            constexpr uint32_t TU = C::TILE_BYTES >> 4, PU = C::PANEL_BYTES >> 4;
-            auto issue_s = [&](int x, int st) {
+            const uint32_t tS = tmem + C::TM_S + x * 128, tO = tmem + C::TM_O + x * D;
+            const uint32_t tP = tmem + C::TM_P + x * C::P_STRIDE;
+            auto issue_s = [&](int st) {
+                const uint32_t kb = k_lo + st * TU;
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * PU + (k % 4) * 2;
-                    mma_ss_lo(tmem + C::TM_S + x * 128, q_lo + x * TU + off, k_lo + st * TU + off,
-                              IDESC_S, k > 0);
+                    mma_ss_lo(tS, q_lo + off, kb + off, IDESC_S, k > 0);
                 }
+                tc_commit(BAR(B_SFULL + x));
+                tc_commit(BAR(B_KEMPTY + st));
             };
-            auto issue_pv = [&](int x, int st, bool acc) {
+            auto issue_pv = [&](int st, bool acc) {
+                const uint32_t vb = v_lo + st * TU;
+                mma_ts_lo(tO, tP, vb, IDESC_O, acc);
 #pragma unroll
-                for (int k = 0; k < BN / 16; ++k)
-                    mma_ts_lo(tmem + C::TM_O + x * D, tmem + C::TM_S + x * 128 + k * 8,
-                              v_lo + st * TU + k * 128, IDESC_O, acc || k > 0);
+                for (int k = 1; k < BN / 16; ++k)
+                    mma_ts_lo(tO, tP + k * 8, vb + k * 128, IDESC_O, 1);
+                tc_commit(BAR(B_PVDONE + x));
+                tc_commit(BAR(B_VEMPTY + st));
             };
             bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag) &&
                       mbar_wait(BAR(B_KFULL + 0), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
-                for (int x = 0; x < ntile; ++x) {
-                    issue_s(x, 0);
-                    tc_commit(BAR(B_SFULL + x));
-                }
-                tc_commit(BAR(B_KEMPTY + 0));
+                issue_s(0);
             }
             for (int j = 0; ok && j < cnt; ++j) {
                 const int st = j % NS, ph = (j / NS) & 1;
                 const int nst = (j + 1) % NS, nph = ((j + 1) / NS) & 1;
                 const bool more = j + 1 < cnt;
-                ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
-                if (ok && more)
-                    ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag);
-                for (int x = 0; ok && x < ntile; ++x) {
-                    ok = mbar_wait(BAR(B_PFULL + x), j & 1, abort_flag);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    issue_pv(x, st, j > 0);
-                    if (x == ntile - 1)
-                        tc_commit(BAR(B_VEMPTY + st));
+                if constexpr (C::P_SEPARATE) {
+                    // S(j+1) as soon as the softmax warps hold S(j) in registers
                     if (more) {
-                        issue_s(x, nst);
-                        tc_commit(BAR(B_SFULL + x));
-                        if (x == ntile - 1)
-                            tc_commit(BAR(B_KEMPTY + nst));
-                    } else {
-                        tc_commit(BAR(B_ODONE + x));
+                        ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag) &&
+                             mbar_wait(BAR(B_SREAD + x), j & 1, abort_flag);
+                        if (!ok)
+                            break;
+                        tc_fence_after();
+                        issue_s(nst);
+                    }
+                }
+                ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag) &&
+                     mbar_wait(BAR(B_PFULL + x), j & 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                issue_pv(st, j > 0);
+                if constexpr (!C::P_SEPARATE) {
+                    // P overwrote S(j): S(j+1) can only follow the P V product that reads it
+                    if (more) {
+                        ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag);
+                        if (!ok)
+                            break;
+                        issue_s(nst);
                     }
                 }
             }
@@ -232,11 +274,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_sel + C::TM_S + x * 128;
         const uint32_t tO = tmem + lane_sel + C::TM_O + x * D;
+        const uint32_t tP = tmem + lane_sel + C::TM_P + x * C::P_STRIDE;
         float m = -CUDART_INF_F, l = 0.f;
         bool ok = true;
+        int cls_nxt = cnt > 0 ? klist[0].y >> 16 : 0;
         for (int j = 0; j < cnt; ++j) {
             const int st = j % NS, ph = (j / NS) & 1;
-            const int cls = klist[j].y >> 16;
+            const int cls = cls_nxt;
+            if (j + 1 < cnt)
+                cls_nxt = klist[j + 1].y >> 16; // used one key tile later
             ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL + x), j & 1, abort_flag));
             if (!ok)
                 break;
@@ -246,6 +292,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             for (int c = 0; c < 4; ++c)
                 tmem_ld32(tS + c * 32, xr[c]);
             tmem_wait_ld();
+            // S(j) is in registers: its columns may be overwritten by S(j+1)
+            tc_fence_before();
+            mbar_arrive(BAR(B_SREAD + x));
             if (cls != TILE_FULL) {
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
                 if (!ok)
@@ -273,6 +322,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (j == 0) {
                 m = m_new;
             } else {
+                // P V of the previous key tile must be done before O or P are touched
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_PVDONE + x), (j - 1) & 1, abort_flag));
+                if (!ok)
+                    break;
+                tc_fence_after();
                 // Rescale the running output only when the maximum grew by more than 2^8; until
                 // then the stale maximum keeps every probability below 256.
                 const bool grow = m_new > m + 8.f;
@@ -308,7 +362,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     sum += p0 + p1;
                     pk[i] = pack_bf16x2(p0, p1);
                 }
-                tmem_st32(tS + c * 32, pk);
+                tmem_st32(tP + c * 32, pk);
             }
             l += sum;
             tmem_wait_st();
@@ -324,7 +378,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     dst[i] = z;
                 P.LSE[(size_t)h * P.T + row] = -CUDART_INF_F;
             }
-        } else if (__all_sync(0xffffffffu, ok && mbar_wait(BAR(B_ODONE + x), 0, abort_flag))) {
+        } else if (__all_sync(0xffffffffu,
+                              ok && mbar_wait(BAR(B_PVDONE + x), (cnt - 1) & 1, abort_flag))) {
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
