@@ -116,6 +116,10 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.cmask = c.take<uint16_t>(nch * nk);
     p.ccount = c.take<int>(nch);
     p.bitems = c.take<int4>(nch * nk);
+    p.scount = c.take<int>(nq);
+    p.skt = c.take<int>(nq * MAX_SINGLE);
+    p.sorder = c.take<uint8_t>(nq * MAX_SINGLE);
+    p.scol = c.take<uint8_t>(nq * MAX_SINGLE * BM);
     if (bytes_out)
         *bytes_out = c.off + 256;
 }
@@ -213,6 +217,7 @@ int plan_call(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partit
         return rc;
     carve_plan(c.plan, ctx->plan_buf.ptr, nullptr);
     c.plan.status = ctx->status;
+    c.plan.allow_single = prob->head_dim == 64 ? 1 : 0;
     if (c.plan.n_qt == 0)
         return PEAGLE_OK;
     ctx->launches += launch_plan(c.plan, prob->anchor, prob->depth, prob->K, c.seq_begin, c.seq_end,
@@ -536,6 +541,7 @@ int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,
     int *status = dev_status ? dev_status
                              : reinterpret_cast<int *>(dev->scratch + STATIC_SCRATCH_BYTES - 256);
     c.plan.status = status;
+    c.plan.allow_single = prob->head_dim == 64 ? 1 : 0;
     // The array keeps whatever the previous call left.  The status word is cleared here; the
     // plan's counters are cleared by the first K0 kernel; every other plan field this call
     // reads is written by this call's K0 kernels first.
@@ -764,6 +770,9 @@ int peagle_classify_tiles(peagle_ctx *ctx, const peagle_problem_t *prob,
     CK(cudaStreamSynchronize(nullptr));
     if (c.plan.n_qt > 0 && c.plan.n_kt > 0)
         CK(cudaMemcpy(host_out, c.plan.cls, (size_t)c.plan.n_qt * c.plan.n_kt, cudaMemcpyDeviceToHost));
+    for (size_t i = 0; i < (size_t)c.plan.n_qt * c.plan.n_kt; ++i)
+        if (host_out[i] == TILE_SINGLE)
+            host_out[i] = TILE_PARTIAL; // an internal refinement of PARTIAL
     return PEAGLE_OK;
 }
 

@@ -1058,6 +1058,7 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
             cudaEventRecord(ev1, s);
         ++launches;
     }
+    launches += launch_bwd_single(p, a, s);
     bwd_finish_dq<<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
         a.dq_acc, static_cast<__nv_bfloat16 *>(a.dQ) + (size_t)p.q_begin * a.Hq * D, n_prep);
     return launches + 1;

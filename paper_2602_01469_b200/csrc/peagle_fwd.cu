@@ -35,7 +35,29 @@ struct FwdParams {
     int Hq, Hkv;
     int two; // 1: two heads per CTA
     float scale_log2;
+    // SINGLE tiles (one allowed key per row), handled pair by pair before the tile loop
+    const int *scount, *skt;
+    const uint8_t *sorder, *scol;
+    const int2 *ktile;
+    const __nv_bfloat16 *Q, *K, *V;
 };
+
+// <a, b> of two rows of 64 bf16 held as 32 packed pairs; products are exact in fp32.
+__device__ __forceinline__ float dot64_bf16(const uint32_t (&a)[32], const uint4 *b)
+{
+    float acc = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const uint4 v = b[i];
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            acc = fmaf(__uint_as_float(a[4 * i + k] << 16), __uint_as_float(w[k] << 16), acc);
+            acc = fmaf(__uint_as_float(a[4 * i + k] & 0xffff0000u), __uint_as_float(w[k] & 0xffff0000u), acc);
+        }
+    }
+    return acc;
+}
 
 template <int D>
 struct FwdCfg {
@@ -93,6 +115,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     const int row0 = P.q_begin + qt * BM;
     const int cnt = P.kcount[qt];
     const int2 *klist = P.klist + (size_t)qt * P.n_kt;
+    // SINGLE tiles exist for head_dim 64 only; their result seeds (m, l, O) before the tile loop
+    const int n_single = (D == 64) ? min(P.scount[qt], MAX_SINGLE) : 0;
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -248,7 +272,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (!ok)
                     break;
                 tc_fence_after();
-                issue_pv(st, j > 0);
+                issue_pv(st, j > 0 || n_single > 0);
                 if constexpr (!C::P_SEPARATE) {
                     // P overwrote S(j): S(j+1) can only follow the P V product that reads it
                     if (more) {
@@ -277,6 +301,66 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const uint32_t tP = tmem + lane_sel + C::TM_P + x * C::P_STRIDE;
         float m = -CUDART_INF_F, l = 0.f;
         bool ok = true;
+        if constexpr (D == 64) {
+            if (n_single > 0) {
+                // One allowed key per row and tile: scores and the weighted values on the CUDA
+                // cores, as an online softmax over at most MAX_SINGLE keys; the result becomes
+                // the starting (m, l, O) of the tile loop.
+                uint32_t qv[32];
+                {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(
+                        P.Q + ((size_t)(row_ok ? row : P.q_begin) * P.Hq + h) * D);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const uint4 v = src[i];
+                        qv[4 * i] = v.x;
+                        qv[4 * i + 1] = v.y;
+                        qv[4 * i + 2] = v.z;
+                        qv[4 * i + 3] = v.w;
+                    }
+                }
+                float o[64];
+#pragma unroll
+                for (int i = 0; i < 64; ++i)
+                    o[i] = 0.f;
+                for (int i = 0; i < n_single; ++i) {
+                    const int slot = P.sorder[qt * MAX_SINGLE + i];
+                    const int col = P.scol[((size_t)qt * MAX_SINGLE + slot) * BM + r];
+                    if (col == NO_COL || !row_ok)
+                        continue;
+                    const size_t tok = (size_t)P.ktile[P.skt[qt * MAX_SINGLE + slot]].x + col;
+                    const float s2 =
+                        dot64_bf16(qv, reinterpret_cast<const uint4 *>(P.K + (tok * P.Hkv + g) * D)) *
+                        P.scale_log2;
+                    const float m_new = fmaxf(m, s2);
+                    const float alpha = fast_exp2(m - m_new); // 0 on the first key (m = -inf)
+                    const float pr = fast_exp2(s2 - m_new);
+                    l = l * alpha + pr;
+                    m = m_new;
+                    const uint4 *vs = reinterpret_cast<const uint4 *>(P.V + (tok * P.Hkv + g) * D);
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 v = vs[c];
+                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            o[8 * c + 2 * k] = fmaf(o[8 * c + 2 * k], alpha, pr * __uint_as_float(w[k] << 16));
+                            o[8 * c + 2 * k + 1] =
+                                fmaf(o[8 * c + 2 * k + 1], alpha, pr * __uint_as_float(w[k] & 0xffff0000u));
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 2; ++c) {
+                    uint32_t ov[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        ov[i] = __float_as_uint(o[32 * c + i]);
+                    tmem_st32(tO + c * 32, ov);
+                }
+                tmem_wait_st(); // ordered before the first P V product by the P hand-over below
+            }
+        }
         int cls_nxt = cnt > 0 ? klist[0].y >> 16 : 0;
         for (int j = 0; j < cnt; ++j) {
             const int st = j % NS, ph = (j / NS) & 1;
@@ -319,14 +403,17 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     mx = fmaxf(mx, __uint_as_float(xr[c][i]));
             mx *= P.scale_log2; // scale > 0, so the max commutes with the scaling
             const float m_new = fmaxf(m, mx);
-            if (j == 0) {
+            if (j == 0 && n_single == 0) {
                 m = m_new;
             } else {
                 // P V of the previous key tile must be done before O or P are touched
-                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_PVDONE + x), (j - 1) & 1, abort_flag));
-                if (!ok)
-                    break;
-                tc_fence_after();
+                if (j > 0) {
+                    ok = __all_sync(0xffffffffu,
+                                    mbar_wait(BAR(B_PVDONE + x), (j - 1) & 1, abort_flag));
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                }
                 // Rescale the running output only when the maximum grew by more than 2^8; until
                 // then the stale maximum keeps every probability below 256.
                 const bool grow = m_new > m + 8.f;
@@ -370,7 +457,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mbar_arrive(BAR(B_PFULL + x));
         }
         // ---- epilogue: normalise, store O and LSE
-        if (cnt == 0) {
+        if (cnt == 0 && n_single == 0) {
             if (row_ok) {
                 uint4 z = make_uint4(0, 0, 0, 0);
                 uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
@@ -379,7 +466,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 P.LSE[(size_t)h * P.T + row] = -CUDART_INF_F;
             }
         } else if (__all_sync(0xffffffffu,
-                              ok && mbar_wait(BAR(B_PVDONE + x), (cnt - 1) & 1, abort_flag))) {
+                              ok && (cnt == 0 ||
+                                     mbar_wait(BAR(B_PVDONE + x), (cnt - 1) & 1, abort_flag)))) {
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
@@ -467,6 +555,14 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     P.Hkv = a.Hkv;
     P.two = ((a.Hq / a.Hkv) % 2 == 0) ? 1 : 0;
     P.scale_log2 = a.scale * 1.4426950408889634f;
+    P.scount = p.scount;
+    P.skt = p.skt;
+    P.sorder = p.sorder;
+    P.scol = p.scol;
+    P.ktile = p.ktile;
+    P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
+    P.K = static_cast<const __nv_bfloat16 *>(a.K);
+    P.V = static_cast<const __nv_bfloat16 *>(a.V);
     static bool attr_set = false;
     if (!attr_set) {
         if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -15,7 +15,12 @@ constexpr int BWD_CQ = 8;        // query tiles per backward work item (aligned 
 constexpr int32_t META_NONE_Q = -1;         // packed metadata of a row outside the partition (sees nothing)
 constexpr int32_t META_NONE_K = 0x7fffffff; // packed metadata of a key outside the batch (seen by nobody)
 
-enum TileClass : uint8_t { TILE_SKIP = 0, TILE_PARTIAL = 1, TILE_FULL = 2 };
+// TILE_SINGLE is internal: a PARTIAL tile in which every query row allows at most one key (the
+// chain tiles of the depth-major layout: one allowed pair per row).  Such tiles are taken out of
+// the tensor-core lists and handled pair by pair.  The test hook reports them as PARTIAL.
+enum TileClass : uint8_t { TILE_SKIP = 0, TILE_PARTIAL = 1, TILE_FULL = 2, TILE_SINGLE = 3 };
+constexpr int MAX_SINGLE = 16;   // SINGLE tiles kept per query tile; further ones stay PARTIAL
+constexpr int NO_COL = 255;      // "this row allows no key of the tile"
 
 // Visible key ranges of one call, passed to kernels by value.
 struct RangeList {
@@ -43,6 +48,11 @@ struct Plan {
     uint16_t *cmask;       // [n_ch][n_kt] per chunk of BWD_CQ query tiles: bit b not skipped, bit 8+b FULL
     int *ccount;           // [n_ch] key tiles with a non-zero word
     int4 *bitems;          // [n_ch * n_kt] backward work items (key tile, chunk, mask word, query tiles)
+    int allow_single;      // 1: the kernels of this head_dim take SINGLE tiles
+    int *scount;           // [n_qt] SINGLE tiles found per query tile (may exceed MAX_SINGLE: clamp)
+    int *skt;              // [n_qt][MAX_SINGLE] key tile of a slot
+    uint8_t *sorder;       // [n_qt][MAX_SINGLE] slots by ascending key tile
+    uint8_t *scol;         // [n_qt][MAX_SINGLE][BM] per row: the one allowed key column, or NO_COL
     int *status;           // device status word
 };
 
@@ -84,6 +94,8 @@ int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cud
                cudaEvent_t ev0, cudaEvent_t ev1);
 int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
                cudaEvent_t ev0, cudaEvent_t ev1);
+// Backward of the SINGLE tiles (adds to the dQ staging and to dK_acc / dV_acc); launches counted.
+int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s);
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s);
 

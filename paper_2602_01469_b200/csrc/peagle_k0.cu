@@ -42,6 +42,9 @@ __global__ void k0_prepare(Plan p, const int32_t *__restrict__ anchor,
         for (int i = 0; i < 8; ++i)
             p.counters[i] = 0;
     }
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < p.n_qt)
+        p.scount[i] = 0;
 }
 
 // ---- 2. tile summaries -----------------------------------------------------------------
@@ -126,7 +129,7 @@ __global__ void k0_classify_quick(Plan p)
 __global__ void k0_classify_exact(Plan p)
 {
     __shared__ int mk[BN];
-    __shared__ int total;
+    __shared__ int total, most, slot;
     const int n = p.counters[0];
     for (int w = blockIdx.x; w < n; w += gridDim.x) {
         const int idx = p.undecided[w];
@@ -135,29 +138,51 @@ __global__ void k0_classify_exact(Plan p)
         const int r0 = p.q_begin + qt * BM, r1 = min(r0 + BM, p.q_end);
         __syncthreads();
         mk[threadIdx.x] = ((int)threadIdx.x < ktile.y) ? p.meta[ktile.x + threadIdx.x] : META_NONE_K;
-        if (threadIdx.x == 0)
+        if (threadIdx.x == 0) {
             total = 0;
+            most = 0;
+            slot = -1;
+        }
         __syncthreads();
-        int cnt = 0;
+        int mine = 0, col = NO_COL;
         if (r0 + (int)threadIdx.x < r1) {
             const int mq = p.meta[r0 + threadIdx.x];
             if (mq != META_NONE_K)
                 for (int c = 0; c < BN; ++c)
-                    cnt += allowed_packed(mq, mk[c]);
+                    if (allowed_packed(mq, mk[c])) {
+                        ++mine;
+                        col = c;
+                    }
         }
-        for (int o = 16; o > 0; o >>= 1)
+        int cnt = mine, mx = mine;
+        for (int o = 16; o > 0; o >>= 1) {
             cnt += __shfl_xor_sync(0xffffffffu, cnt, o);
-        if ((threadIdx.x & 31) == 0)
+            mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        if ((threadIdx.x & 31) == 0) {
             atomicAdd(&total, cnt);
+            atomicMax(&most, mx);
+        }
         __syncthreads();
         if (threadIdx.x == 0) {
             uint8_t c = TILE_PARTIAL;
-            if (total == 0)
+            if (total == 0) {
                 c = TILE_SKIP;
-            else if (ktile.y == BN && total == (r1 - r0) * BN)
+            } else if (ktile.y == BN && total == (r1 - r0) * BN) {
                 c = TILE_FULL;
+            } else if (p.allow_single && most <= 1) {
+                const int sl = atomicAdd(&p.scount[qt], 1);
+                if (sl < MAX_SINGLE) {
+                    c = TILE_SINGLE;
+                    slot = sl;
+                    p.skt[qt * MAX_SINGLE + sl] = kt;
+                }
+            }
             p.cls[idx] = c;
         }
+        __syncthreads();
+        if (slot >= 0)
+            p.scol[((size_t)qt * MAX_SINGLE + slot) * BM + threadIdx.x] = (uint8_t)col;
     }
 }
 
@@ -176,6 +201,8 @@ __global__ void k0_lists(Plan p)
         uint8_t c = TILE_SKIP;
         if (o < p.n_kt)
             c = p.cls[(size_t)self * p.n_kt + o];
+        if (c == TILE_SINGLE)
+            c = TILE_SKIP; // handled outside the tensor-core lists
         const unsigned bal = __ballot_sync(0xffffffffu, c != TILE_SKIP);
         const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
         if (lane == 0)
@@ -194,8 +221,24 @@ __global__ void k0_lists(Plan p)
             base += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
         __syncthreads();
     }
-    if (threadIdx.x == 0)
+    if (threadIdx.x == 0) {
         p.kcount[self] = base;
+        // SINGLE slots were handed out in arrival order: list them by ascending key tile so that
+        // the order of the per-pair sums does not change from run to run
+        const int ns = min(p.scount[self], MAX_SINGLE);
+        uint8_t ord[MAX_SINGLE];
+        for (int i = 0; i < ns; ++i) {
+            int j = i;
+            const int kt = p.skt[self * MAX_SINGLE + i];
+            while (j > 0 && p.skt[self * MAX_SINGLE + ord[j - 1]] > kt) {
+                ord[j] = ord[j - 1];
+                --j;
+            }
+            ord[j] = (uint8_t)i;
+        }
+        for (int i = 0; i < ns; ++i)
+            p.sorder[self * MAX_SINGLE + i] = ord[i];
+    }
 }
 
 // ---- 4b. order query tiles longest-first ----------------------------------------------------
@@ -241,7 +284,7 @@ __global__ void k0_chunk_masks(Plan p)
             const int qt = c * BWD_CQ + b;
             if (qt < p.n_qt) {
                 const uint8_t cl = p.cls[(size_t)qt * p.n_kt + kt];
-                if (cl != TILE_SKIP)
+                if (cl != TILE_SKIP && cl != TILE_SINGLE)
                     m |= 1u << b;
                 if (cl == TILE_FULL)
                     m |= 1u << (8 + b);
