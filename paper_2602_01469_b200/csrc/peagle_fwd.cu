@@ -36,9 +36,8 @@ struct FwdParams {
     int two; // 1: two heads per CTA
     float scale_log2;
     // SINGLE tiles (one allowed key per row), handled pair by pair before the tile loop
-    const int *scount, *skt;
-    const uint8_t *sorder, *scol;
-    const int2 *ktile;
+    const int *scount;
+    const int32_t *stok; // [n_qt][MAX_SINGLE][BM] key token of entry i for row r, or -1
     const __nv_bfloat16 *Q, *K, *V;
 };
 
@@ -319,37 +318,52 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         qv[4 * i + 3] = v.w;
                     }
                 }
+                // pass 1: the keys of this row and their scores (loads of different keys are
+                // independent, so their latencies overlap)
+                size_t tok[MAX_SINGLE];
+                float sc[MAX_SINGLE];
+#pragma unroll
+                for (int i = 0; i < MAX_SINGLE; ++i) {
+                    sc[i] = -CUDART_INF_F;
+                    tok[i] = 0;
+                    if (i < n_single) {
+                        const int t = P.stok[((size_t)qt * MAX_SINGLE + i) * BM + r];
+                        if (t >= 0 && row_ok) {
+                            tok[i] = (size_t)t * P.Hkv + g;
+                            sc[i] = 0.f;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < MAX_SINGLE; ++i)
+                    if (i < n_single && sc[i] == 0.f) {
+                        sc[i] = dot64_bf16(qv, reinterpret_cast<const uint4 *>(P.K + tok[i] * D)) *
+                                P.scale_log2;
+                        m = fmaxf(m, sc[i]);
+                    }
+                // pass 2: probabilities against the known maximum, weighted values
                 float o[64];
 #pragma unroll
                 for (int i = 0; i < 64; ++i)
                     o[i] = 0.f;
-                for (int i = 0; i < n_single; ++i) {
-                    const int slot = P.sorder[qt * MAX_SINGLE + i];
-                    const int col = P.scol[((size_t)qt * MAX_SINGLE + slot) * BM + r];
-                    if (col == NO_COL || !row_ok)
-                        continue;
-                    const size_t tok = (size_t)P.ktile[P.skt[qt * MAX_SINGLE + slot]].x + col;
-                    const float s2 =
-                        dot64_bf16(qv, reinterpret_cast<const uint4 *>(P.K + (tok * P.Hkv + g) * D)) *
-                        P.scale_log2;
-                    const float m_new = fmaxf(m, s2);
-                    const float alpha = fast_exp2(m - m_new); // 0 on the first key (m = -inf)
-                    const float pr = fast_exp2(s2 - m_new);
-                    l = l * alpha + pr;
-                    m = m_new;
-                    const uint4 *vs = reinterpret_cast<const uint4 *>(P.V + (tok * P.Hkv + g) * D);
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        const uint4 v = vs[c];
-                        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                for (int i = 0; i < MAX_SINGLE; ++i)
+                    if (i < n_single && sc[i] != -CUDART_INF_F) {
+                        const float pr = fast_exp2(sc[i] - m);
+                        l += pr;
+                        const uint4 *vs = reinterpret_cast<const uint4 *>(P.V + tok[i] * D);
 #pragma unroll
-                        for (int k = 0; k < 4; ++k) {
-                            o[8 * c + 2 * k] = fmaf(o[8 * c + 2 * k], alpha, pr * __uint_as_float(w[k] << 16));
-                            o[8 * c + 2 * k + 1] =
-                                fmaf(o[8 * c + 2 * k + 1], alpha, pr * __uint_as_float(w[k] & 0xffff0000u));
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 v = vs[c];
+                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                o[8 * c + 2 * k] = fmaf(pr, __uint_as_float(w[k] << 16), o[8 * c + 2 * k]);
+                                o[8 * c + 2 * k + 1] =
+                                    fmaf(pr, __uint_as_float(w[k] & 0xffff0000u), o[8 * c + 2 * k + 1]);
+                            }
                         }
                     }
-                }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t ov[32];
@@ -556,10 +570,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     P.two = ((a.Hq / a.Hkv) % 2 == 0) ? 1 : 0;
     P.scale_log2 = a.scale * 1.4426950408889634f;
     P.scount = p.scount;
-    P.skt = p.skt;
-    P.sorder = p.sorder;
-    P.scol = p.scol;
-    P.ktile = p.ktile;
+    P.stok = p.stok;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);

@@ -5,11 +5,10 @@
 // Delta = <dO, O> (Section 3.2's backward, same formulas as the tile kernel):
 //   s = <Q[q,h], K[k]>,  p = exp(scale * s - LSE),  dp = <dO[q,h], V[k]>,  ds = p * (dp - Delta)
 //   dQ[q,h] += scale * ds * K[k]      dK[k] += scale * ds * Q[q,h]      dV[k] += p * dO[q,h]
-// Two kernels, both query-major so that no reverse (key -> queries) list is needed:
-//   single_dq   one thread per (query row, head): dQ over the row's SINGLE keys, one fp32 add to
-//               the dQ staging row;
-//   single_dkv  one thread per (query row, SINGLE slot, KV head): dK / dV of the row's key summed
-//               over the heads of the group in registers, one fp32 add per key row.
+// One kernel, query-major so that no reverse (key -> queries) list is needed: eight lanes per
+// (query row, KV head) hold 8 of the 64 elements each; for every head of the group they form the
+// row's dQ (one fp32 add to the staging row per head) and add into per-key dK / dV sums kept in
+// registers across the heads (one fp32 add per key row at the end).
 #include <math_constants.h>
 
 #include "peagle_internal.h"
@@ -19,9 +18,8 @@ namespace peagle {
 using namespace sm100;
 
 struct SingleParams {
-    const int *scount, *skt;
-    const uint8_t *sorder, *scol;
-    const int2 *ktile;
+    const int *scount;
+    const int32_t *stok; // [n_qt][MAX_SINGLE][BM]
     const __nv_bfloat16 *Q, *K, *V, *dO;
     const float *nl2, *nd; // [Hq][q_pad]
     float *dq_acc, *dK_acc, *dV_acc;
@@ -29,137 +27,108 @@ struct SingleParams {
     float scale, scale_log2;
 };
 
-__device__ __forceinline__ void load_row64(const __nv_bfloat16 *src, uint32_t (&v)[32])
+// A row of 64 bf16 is spread over 8 consecutive lanes, 8 elements (one 16-byte load) per lane, so
+// that a warp reads four whole rows with every load and dot products finish with three shuffles.
+struct Chunk {
+    float v[8];
+};
+__device__ __forceinline__ Chunk load_chunk(const __nv_bfloat16 *row, int sub)
 {
-    const uint4 *s4 = reinterpret_cast<const uint4 *>(src);
+    const uint4 t = reinterpret_cast<const uint4 *>(row)[sub];
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+    Chunk c;
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        const uint4 t = s4[i];
-        v[4 * i] = t.x;
-        v[4 * i + 1] = t.y;
-        v[4 * i + 2] = t.z;
-        v[4 * i + 3] = t.w;
+    for (int i = 0; i < 4; ++i) {
+        c.v[2 * i] = __uint_as_float(w[i] << 16);
+        c.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
     }
+    return c;
 }
-__device__ __forceinline__ float lo_bf16(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float hi_bf16(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-__device__ __forceinline__ float dot64(const uint32_t (&a)[32], const uint32_t (&b)[32])
+__device__ __forceinline__ void red_chunk(float *dst, const float (&x)[8], float f)
 {
-    float acc = 0.f;
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        acc = fmaf(lo_bf16(a[i]), lo_bf16(b[i]), acc);
-        acc = fmaf(hi_bf16(a[i]), hi_bf16(b[i]), acc);
-    }
-    return acc;
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x[0] * f),
+                 "f"(x[1] * f), "f"(x[2] * f), "f"(x[3] * f)
+                 : "memory");
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4), "f"(x[4] * f),
+                 "f"(x[5] * f), "f"(x[6] * f), "f"(x[7] * f)
+                 : "memory");
 }
 
-// Thread (row r of the partition, head h); threads of a block share the row's query tile.
-__global__ void __launch_bounds__(128) single_dq(const SingleParams P)
+// Unit (row r of the partition, KV head g) = 8 lanes; a block of 128 threads holds 16 units.
+// Keys are taken KEYS at a time so that their dK / dV sums fit in registers.
+__global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
 {
-    const int per_row = P.Hq;
-    const size_t gid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int r = (int)(gid / per_row), h = (int)(gid % per_row);
+    constexpr int KEYS = 8;
+    const int sub = threadIdx.x & 7;
+    const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
+    const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
+    const int r = (int)(unit / P.Hkv), g = (int)(unit % P.Hkv);
     const int row = P.q_begin + r;
     if (row >= P.q_end)
-        return;
+        return; // the 8 lanes of a unit leave together
     const int qt = r / BM, rr = r % BM;
     const int ns = min(P.scount[qt], MAX_SINGLE);
-    if (ns == 0)
-        return;
-    const int g = h / (P.Hq / P.Hkv);
-    const float nl2 = P.nl2[(size_t)h * P.q_pad + r], nd = P.nd[(size_t)h * P.q_pad + r];
-    uint32_t q[32], dO[32];
-    load_row64(P.Q + ((size_t)row * P.Hq + h) * 64, q);
-    load_row64(P.dO + ((size_t)row * P.Hq + h) * 64, dO);
-    float dq[64];
-#pragma unroll
-    for (int i = 0; i < 64; ++i)
-        dq[i] = 0.f;
-    bool any = false;
-    for (int i = 0; i < ns; ++i) {
-        const int slot = P.sorder[qt * MAX_SINGLE + i];
-        const int col = P.scol[((size_t)qt * MAX_SINGLE + slot) * BM + rr];
-        if (col == NO_COL)
-            continue;
-        any = true;
-        const size_t tok = (size_t)P.ktile[P.skt[qt * MAX_SINGLE + slot]].x + col;
-        uint32_t k[32], v[32];
-        load_row64(P.K + (tok * P.Hkv + g) * 64, k);
-        load_row64(P.V + (tok * P.Hkv + g) * 64, v);
-        const float p = fast_exp2(fmaf(dot64(q, k), P.scale_log2, nl2)); // nl2 = -inf: p = 0
-        const float ds = p * (dot64(dO, v) + nd);
-#pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            dq[2 * c] = fmaf(ds, lo_bf16(k[c]), dq[2 * c]);
-            dq[2 * c + 1] = fmaf(ds, hi_bf16(k[c]), dq[2 * c + 1]);
-        }
-    }
-    if (!any)
-        return;
-    float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * 64;
-#pragma unroll
-    for (int c = 0; c < 64; c += 4)
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + c),
-                     "f"(dq[c] * P.scale), "f"(dq[c + 1] * P.scale), "f"(dq[c + 2] * P.scale),
-                     "f"(dq[c + 3] * P.scale)
-                     : "memory");
-}
-
-// Block (query tile qt, slot index i, KV head g), thread = row of the tile.
-__global__ void __launch_bounds__(128) single_dkv(const SingleParams P)
-{
-    const int g = blockIdx.x % P.Hkv;
-    const int i = (blockIdx.x / P.Hkv) % MAX_SINGLE;
-    const int qt = blockIdx.x / (P.Hkv * MAX_SINGLE);
-    if (i >= min(P.scount[qt], MAX_SINGLE))
-        return;
-    const int rr = threadIdx.x, r = qt * BM + rr, row = P.q_begin + r;
-    if (row >= P.q_end)
-        return;
-    const int slot = P.sorder[qt * MAX_SINGLE + i];
-    const int col = P.scol[((size_t)qt * MAX_SINGLE + slot) * BM + rr];
-    if (col == NO_COL)
-        return;
-    const size_t tok = (size_t)P.ktile[P.skt[qt * MAX_SINGLE + slot]].x + col;
-    uint32_t k[32], v[32];
-    load_row64(P.K + (tok * P.Hkv + g) * 64, k);
-    load_row64(P.V + (tok * P.Hkv + g) * 64, v);
-    float dk[64], dv[64];
-#pragma unroll
-    for (int c = 0; c < 64; ++c) {
-        dk[c] = 0.f;
-        dv[c] = 0.f;
-    }
     const int G = P.Hq / P.Hkv;
-    for (int hh = 0; hh < G; ++hh) {
-        const int h = g * G + hh;
-        const float nl2 = P.nl2[(size_t)h * P.q_pad + r], nd = P.nd[(size_t)h * P.q_pad + r];
-        uint32_t t[32];
-        load_row64(P.Q + ((size_t)row * P.Hq + h) * 64, t);
-        const float s = dot64(t, k);
-        const float p = fast_exp2(fmaf(s, P.scale_log2, nl2));
-        uint32_t u[32];
-        load_row64(P.dO + ((size_t)row * P.Hq + h) * 64, u);
-        const float ds = p * (dot64(u, v) + nd);
+    for (int i0 = 0; i0 < ns; i0 += KEYS) {
+        int tok[KEYS];
+        bool any = false;
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            dk[2 * c] = fmaf(ds, lo_bf16(t[c]), dk[2 * c]);
-            dk[2 * c + 1] = fmaf(ds, hi_bf16(t[c]), dk[2 * c + 1]);
-            dv[2 * c] = fmaf(p, lo_bf16(u[c]), dv[2 * c]);
-            dv[2 * c + 1] = fmaf(p, hi_bf16(u[c]), dv[2 * c + 1]);
+        for (int i = 0; i < KEYS; ++i) {
+            tok[i] = (i0 + i < ns) ? P.stok[((size_t)qt * MAX_SINGLE + i0 + i) * BM + rr] : -1;
+            any |= tok[i] >= 0;
         }
-    }
-    float *dkd = P.dK_acc + (tok * P.Hkv + g) * 64, *dvd = P.dV_acc + (tok * P.Hkv + g) * 64;
+        if (!any)
+            continue;
+        float dk[KEYS][8], dv[KEYS][8];
 #pragma unroll
-    for (int c = 0; c < 64; c += 4) {
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dkd + c),
-                     "f"(dk[c] * P.scale), "f"(dk[c + 1] * P.scale), "f"(dk[c + 2] * P.scale),
-                     "f"(dk[c + 3] * P.scale)
-                     : "memory");
-        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dvd + c), "f"(dv[c]),
-                     "f"(dv[c + 1]), "f"(dv[c + 2]), "f"(dv[c + 3])
-                     : "memory");
+        for (int i = 0; i < KEYS; ++i)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                dk[i][e] = 0.f;
+                dv[i][e] = 0.f;
+            }
+        for (int hh = 0; hh < G; ++hh) {
+            const int h = g * G + hh;
+            const float nl2 = P.nl2[(size_t)h * P.q_pad + r], nd = P.nd[(size_t)h * P.q_pad + r];
+            const Chunk q = load_chunk(P.Q + ((size_t)row * P.Hq + h) * 64, sub);
+            const Chunk dO = load_chunk(P.dO + ((size_t)row * P.Hq + h) * 64, sub);
+            float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < KEYS; ++i) {
+                if (tok[i] < 0)
+                    continue; // same for the 8 lanes of the unit
+                const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64;
+                const Chunk k = load_chunk(P.K + kr, sub); // re-read per head: stays in L1
+                const Chunk v = load_chunk(P.V + kr, sub);
+                float s = 0.f, dp = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    s = fmaf(q.v[e], k.v[e], s);
+                    dp = fmaf(dO.v[e], v.v[e], dp);
+                }
+#pragma unroll
+                for (int o = 1; o < 8; o <<= 1) {
+                    s += __shfl_xor_sync(um, s, o);
+                    dp += __shfl_xor_sync(um, dp, o);
+                }
+                const float p = fast_exp2(fmaf(s, P.scale_log2, nl2)); // nl2 = -inf: p = 0
+                const float ds = p * (dp + nd);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    dq[e] = fmaf(ds, k.v[e], dq[e]);
+                    dk[i][e] = fmaf(ds, q.v[e], dk[i][e]);
+                    dv[i][e] = fmaf(p, dO.v[e], dv[i][e]);
+                }
+            }
+            red_chunk(P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8, dq, P.scale);
+        }
+#pragma unroll
+        for (int i = 0; i < KEYS; ++i)
+            if (tok[i] >= 0) {
+                const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64 + sub * 8;
+                red_chunk(P.dK_acc + kr, dk[i], P.scale);
+                red_chunk(P.dV_acc + kr, dv[i], 1.f);
+            }
     }
 }
 
@@ -169,10 +138,7 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
         return 0;
     SingleParams P;
     P.scount = p.scount;
-    P.skt = p.skt;
-    P.sorder = p.sorder;
-    P.scol = p.scol;
-    P.ktile = p.ktile;
+    P.stok = p.stok;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);
@@ -190,10 +156,9 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.Hkv = a.Hkv;
     P.scale = a.scale;
     P.scale_log2 = a.scale * 1.4426950408889634f;
-    const size_t n_dq = (size_t)(p.q_end - p.q_begin) * a.Hq;
-    single_dq<<<(unsigned)((n_dq + 127) / 128), 128, 0, s>>>(P);
-    single_dkv<<<(unsigned)((size_t)p.n_qt * MAX_SINGLE * a.Hkv), 128, 0, s>>>(P);
-    return 2;
+    const size_t units = (size_t)(p.q_end - p.q_begin) * a.Hkv; // of 8 lanes each
+    single_bwd<<<(unsigned)((units + 15) / 16), 128, 0, s>>>(P);
+    return 1;
 }
 
 } // namespace peagle
