@@ -121,6 +121,7 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.sorder = c.take<uint8_t>(nq * MAX_SINGLE);
     p.scol = c.take<uint8_t>(nq * MAX_SINGLE * BM);
     p.stok = c.take<int32_t>(nq * MAX_SINGLE * BM);
+    p.sbase = c.take<int>(nq * MAX_SINGLE);
     if (bytes_out)
         *bytes_out = c.off + 256;
 }

@@ -38,6 +38,7 @@ struct FwdParams {
     // SINGLE tiles (one allowed key per row), handled pair by pair before the tile loop
     const int *scount;
     const int32_t *stok; // [n_qt][MAX_SINGLE][BM] key token of entry i for row r, or -1
+    const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
     const __nv_bfloat16 *Q, *K, *V;
 };
 
@@ -148,7 +149,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         reg_dec<56>();
     if (warp == 9) {
         // ------------------------------------------------------------ producer
-        if (cnt > 0) {
+        if (cnt > 0 || n_single > 0) {
             if (lane == 0) {
                 tma_prefetch_desc(&tmQ);
                 tma_prefetch_desc(&tmK);
@@ -158,6 +159,29 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     for (int pn = 0; pn < C::PANELS; ++pn)
                         tma_load_3d(sb + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmQ,
                                     BAR(B_QFULL), pn * 64, h0 + x, row0);
+            }
+            // The key tiles of the SINGLE entries go through the same K / V ring first; the softmax
+            // warps read their rows from shared memory.
+            bool live = true;
+            for (int i = 0; live && i < n_single; ++i) {
+                const int st = i % NS, ph = (i / NS) & 1;
+                const int start = P.sbase[qt * MAX_SINGLE + i];
+                bool ok = true;
+                if (lane == 0) {
+                    ok = mbar_wait(BAR(B_KEMPTY + st), ph ^ 1, abort_flag) &&
+                         mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, abort_flag);
+                    if (ok) {
+                        mbar_arrive_expect_tx(BAR(B_KFULL + st), C::TILE_BYTES);
+                        mbar_arrive_expect_tx(BAR(B_VFULL + st), C::TILE_BYTES);
+                        for (int pn = 0; pn < C::PANELS; ++pn) {
+                            tma_load_3d(sb + C::OFF_K + st * C::TILE_BYTES + pn * C::PANEL_BYTES,
+                                        &tmK, BAR(B_KFULL + st), pn * 64, g, start);
+                            tma_load_3d(sb + C::OFF_V + st * C::TILE_BYTES + pn * C::PANEL_BYTES,
+                                        &tmV, BAR(B_VFULL + st), pn * 64, g, start);
+                        }
+                    }
+                }
+                live = __all_sync(0xffffffffu, ok);
             }
             // List entries and key metadata are fetched one key tile ahead, so that no global
             // load latency sits between a stage becoming free and its TMA loads.
@@ -170,12 +194,14 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     mv[i] = (need && t < len) ? P.meta[start + t] : META_NONE_K;
                 }
             };
-            int2 e_cur = klist[0];
+            int2 e_cur = cnt > 0 ? klist[0] : make_int2(0, 0);
             int2 e_nxt = cnt > 1 ? klist[1] : e_cur;
             int32_t m_cur[BN / 32], m_nxt[BN / 32];
-            tile_meta(e_cur, m_cur);
-            for (int j = 0; j < cnt; ++j) {
-                const int st = j % NS, ph = (j / NS) & 1;
+            if (cnt > 0)
+                tile_meta(e_cur, m_cur);
+            for (int j = 0; live && j < cnt; ++j) {
+                const int jj = n_single + j; // position in the K / V ring
+                const int st = jj % NS, ph = (jj / NS) & 1;
                 const int start = e_cur.x;
                 const int2 e_nn = j + 2 < cnt ? klist[j + 2] : e_nxt;
                 if (j + 1 < cnt)
@@ -245,15 +271,21 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 tc_commit(BAR(B_PVDONE + x));
                 tc_commit(BAR(B_VEMPTY + st));
             };
-            bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag) &&
-                      mbar_wait(BAR(B_KFULL + 0), 0, abort_flag);
+            // Ring positions: the SINGLE entries come first.  Their phases are waited for one by
+            // one: a parity wait is only meaningful on the phase that follows the last one seen.
+            bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag);
+            for (int i = 0; ok && i < n_single; ++i)
+                ok = mbar_wait(BAR(B_KFULL + i % NS), (i / NS) & 1, abort_flag) &&
+                     mbar_wait(BAR(B_VFULL + i % NS), (i / NS) & 1, abort_flag);
+            ok = ok && mbar_wait(BAR(B_KFULL + n_single % NS), (n_single / NS) & 1, abort_flag);
             if (ok) {
                 tc_fence_after();
-                issue_s(0);
+                issue_s(n_single % NS);
             }
             for (int j = 0; ok && j < cnt; ++j) {
-                const int st = j % NS, ph = (j / NS) & 1;
-                const int nst = (j + 1) % NS, nph = ((j + 1) / NS) & 1;
+                const int jj = n_single + j;
+                const int st = jj % NS, ph = (jj / NS) & 1;
+                const int nst = (jj + 1) % NS, nph = ((jj + 1) / NS) & 1;
                 const bool more = j + 1 < cnt;
                 if constexpr (C::P_SEPARATE) {
                     // S(j+1) as soon as the softmax warps hold S(j) in registers
@@ -302,59 +334,63 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         bool ok = true;
         if constexpr (D == 64) {
             if (n_single > 0) {
-                // One allowed key per row and tile: scores and the weighted values on the CUDA
-                // cores, as an online softmax over at most MAX_SINGLE keys; the result becomes
-                // the starting (m, l, O) of the tile loop.
+                // One allowed key per row and tile: the score and the weighted value on the CUDA
+                // cores, rows read from the staged K / V tiles, as an online softmax; the result
+                // becomes the starting (m, l, O) of the tile loop.
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL), 0, abort_flag));
                 uint32_t qv[32];
                 {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(
-                        P.Q + ((size_t)(row_ok ? row : P.q_begin) * P.Hq + h) * D);
+                    const uint8_t *qrow = sp + C::OFF_Q + x * C::TILE_BYTES + r * 128;
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const uint4 v = src[i];
-                        qv[4 * i] = v.x;
-                        qv[4 * i + 1] = v.y;
-                        qv[4 * i + 2] = v.z;
-                        qv[4 * i + 3] = v.w;
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(qrow + ((c ^ (r & 7)) << 4));
+                        qv[4 * c] = v.x;
+                        qv[4 * c + 1] = v.y;
+                        qv[4 * c + 2] = v.z;
+                        qv[4 * c + 3] = v.w;
                     }
                 }
-                // pass 1: the keys of this row and their scores (loads of different keys are
-                // independent, so their latencies overlap)
-                size_t tok[MAX_SINGLE];
-                float sc[MAX_SINGLE];
-#pragma unroll
-                for (int i = 0; i < MAX_SINGLE; ++i) {
-                    sc[i] = -CUDART_INF_F;
-                    tok[i] = 0;
-                    if (i < n_single) {
-                        const int t = P.stok[((size_t)qt * MAX_SINGLE + i) * BM + r];
-                        if (t >= 0 && row_ok) {
-                            tok[i] = (size_t)t * P.Hkv + g;
-                            sc[i] = 0.f;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < MAX_SINGLE; ++i)
-                    if (i < n_single && sc[i] == 0.f) {
-                        sc[i] = dot64_bf16(qv, reinterpret_cast<const uint4 *>(P.K + tok[i] * D)) *
-                                P.scale_log2;
-                        m = fmaxf(m, sc[i]);
-                    }
-                // pass 2: probabilities against the known maximum, weighted values
                 float o[64];
 #pragma unroll
                 for (int i = 0; i < 64; ++i)
                     o[i] = 0.f;
-#pragma unroll
-                for (int i = 0; i < MAX_SINGLE; ++i)
-                    if (i < n_single && sc[i] != -CUDART_INF_F) {
-                        const float pr = fast_exp2(sc[i] - m);
-                        l += pr;
-                        const uint4 *vs = reinterpret_cast<const uint4 *>(P.V + tok[i] * D);
+                for (int i = 0; ok && i < n_single; ++i) {
+                    const int st = i % NS, ph = (i / NS) & 1;
+                    const int t = P.stok[((size_t)qt * MAX_SINGLE + i) * BM + r];
+                    const int col = t - P.sbase[qt * MAX_SINGLE + i];
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
+                                                     mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
+                    if (!ok)
+                        break;
+                    if (t >= 0 && row_ok) {
+                        const uint8_t *krow = sp + C::OFF_K + st * C::TILE_BYTES + col * 128;
+                        const uint8_t *vrow = sp + C::OFF_V + st * C::TILE_BYTES + col * 128;
+                        float acc = 0.f;
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
-                            const uint4 v = vs[c];
+                            const uint4 v = *reinterpret_cast<const uint4 *>(krow + ((c ^ (col & 7)) << 4));
+                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                acc = fmaf(__uint_as_float(qv[4 * c + k] << 16), __uint_as_float(w[k] << 16), acc);
+                                acc = fmaf(__uint_as_float(qv[4 * c + k] & 0xffff0000u),
+                                           __uint_as_float(w[k] & 0xffff0000u), acc);
+                            }
+                        }
+                        const float s2 = acc * P.scale_log2;
+                        if (s2 > m) { // bring the running sums to the new maximum
+                            const float alpha = fast_exp2(m - s2); // 0 for the first key
+                            l *= alpha;
+#pragma unroll
+                            for (int e = 0; e < 64; ++e)
+                                o[e] *= alpha;
+                            m = s2;
+                        }
+                        const float pr = fast_exp2(s2 - m);
+                        l += pr;
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(vrow + ((c ^ (col & 7)) << 4));
                             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
@@ -364,6 +400,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                             }
                         }
                     }
+                    // every thread of this tile's four warps is done with the stage
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + x) : "memory");
+                    if (r == 0) {
+                        mbar_arrive(BAR(B_KEMPTY + st));
+                        mbar_arrive(BAR(B_VEMPTY + st));
+                    }
+                }
 #pragma unroll
                 for (int c = 0; c < 2; ++c) {
                     uint32_t ov[32];
@@ -376,8 +419,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         }
         int cls_nxt = cnt > 0 ? klist[0].y >> 16 : 0;
-        for (int j = 0; j < cnt; ++j) {
-            const int st = j % NS, ph = (j / NS) & 1;
+        for (int j = 0; ok && j < cnt; ++j) {
+            const int jj = n_single + j; // position in the K / V ring
+            const int st = jj % NS, ph = (jj / NS) & 1;
             const int cls = cls_nxt;
             if (j + 1 < cnt)
                 cls_nxt = klist[j + 1].y >> 16; // used one key tile later
@@ -571,6 +615,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     P.scale_log2 = a.scale * 1.4426950408889634f;
     P.scount = p.scount;
     P.stok = p.stok;
+    P.sbase = p.sbase;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);

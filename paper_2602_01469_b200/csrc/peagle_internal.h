@@ -53,6 +53,7 @@ struct Plan {
     int *skt;              // [n_qt][MAX_SINGLE] key tile of a slot
     uint8_t *sorder;       // [n_qt][MAX_SINGLE] slots by ascending key tile
     uint8_t *scol;         // [n_qt][MAX_SINGLE][BM] per row: the one allowed key column, or NO_COL
+    int *sbase;            // [n_qt][MAX_SINGLE] first token of entry i's key tile
     int32_t *stok;         // [n_qt][MAX_SINGLE][BM] what the kernels read: entry i (slots by ascending
                            // key tile) of row r is the token index of its key, or -1
     int *status;           // device status word

@@ -236,8 +236,10 @@ __global__ void k0_lists(Plan p)
             }
             ord[j] = (uint8_t)i;
         }
-        for (int i = 0; i < ns; ++i)
+        for (int i = 0; i < ns; ++i) {
             p.sorder[self * MAX_SINGLE + i] = ord[i];
+            p.sbase[self * MAX_SINGLE + i] = p.ktile[p.skt[self * MAX_SINGLE + ord[i]]].x;
+        }
     }
     __syncthreads();
     {
