@@ -32,6 +32,17 @@ struct SingleParams {
 struct Chunk {
     float v[8];
 };
+__device__ __forceinline__ Chunk unpack_chunk(const uint4 t)
+{
+    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+    Chunk c;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        c.v[2 * i] = __uint_as_float(w[i] << 16);
+        c.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+    return c;
+}
 __device__ __forceinline__ Chunk load_chunk(const __nv_bfloat16 *row, int sub)
 {
     const uint4 t = reinterpret_cast<const uint4 *>(row)[sub];
@@ -58,7 +69,7 @@ __device__ __forceinline__ void red_chunk(float *dst, const float (&x)[8], float
 // Keys are taken KEYS at a time so that their dK / dV sums fit in registers.
 __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
 {
-    constexpr int KEYS = 8;
+    constexpr int KEYS = 4;
     const int sub = threadIdx.x & 7;
     const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
     const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
@@ -80,26 +91,41 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
         if (!any)
             continue;
         float dk[KEYS][8], dv[KEYS][8];
+        uint4 kp[KEYS], vp[KEYS]; // the keys' elements of this lane, packed bf16
 #pragma unroll
-        for (int i = 0; i < KEYS; ++i)
+        for (int i = 0; i < KEYS; ++i) {
+            const size_t kr = ((size_t)(tok[i] >= 0 ? tok[i] : 0) * P.Hkv + g) * 64;
+            kp[i] = reinterpret_cast<const uint4 *>(P.K + kr)[sub];
+            vp[i] = reinterpret_cast<const uint4 *>(P.V + kr)[sub];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
                 dk[i][e] = 0.f;
                 dv[i][e] = 0.f;
             }
+        }
+        // the rows of the next head are requested before this head's arithmetic
+        const size_t qoff = ((size_t)row * P.Hq + (size_t)g * G) * 64;
+        uint4 qn = reinterpret_cast<const uint4 *>(P.Q + qoff)[sub];
+        uint4 dn = reinterpret_cast<const uint4 *>(P.dO + qoff)[sub];
+        float nl2n = P.nl2[(size_t)(g * G) * P.q_pad + r], ndn = P.nd[(size_t)(g * G) * P.q_pad + r];
         for (int hh = 0; hh < G; ++hh) {
             const int h = g * G + hh;
-            const float nl2 = P.nl2[(size_t)h * P.q_pad + r], nd = P.nd[(size_t)h * P.q_pad + r];
-            const Chunk q = load_chunk(P.Q + ((size_t)row * P.Hq + h) * 64, sub);
-            const Chunk dO = load_chunk(P.dO + ((size_t)row * P.Hq + h) * 64, sub);
+            const float nl2 = nl2n, nd = ndn;
+            const Chunk q = unpack_chunk(qn);
+            const Chunk dO = unpack_chunk(dn);
+            if (hh + 1 < G) {
+                qn = reinterpret_cast<const uint4 *>(P.Q + qoff + (size_t)(hh + 1) * 64)[sub];
+                dn = reinterpret_cast<const uint4 *>(P.dO + qoff + (size_t)(hh + 1) * 64)[sub];
+                nl2n = P.nl2[(size_t)(h + 1) * P.q_pad + r];
+                ndn = P.nd[(size_t)(h + 1) * P.q_pad + r];
+            }
             float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < KEYS; ++i) {
                 if (tok[i] < 0)
                     continue; // same for the 8 lanes of the unit
-                const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64;
-                const Chunk k = load_chunk(P.K + kr, sub); // re-read per head: stays in L1
-                const Chunk v = load_chunk(P.V + kr, sub);
+                const Chunk k = unpack_chunk(kp[i]);
+                const Chunk v = unpack_chunk(vp[i]);
                 float s = 0.f, dp = 0.f;
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
