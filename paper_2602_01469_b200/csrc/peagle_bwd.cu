@@ -440,11 +440,12 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // warps need once per step for the dS^T hand-over.
 struct Bwd64Cfg {
     static constexpr int D = 64;
-    static constexpr int NSQ = 3;
+    static constexpr int NSQ = 2;
     static constexpr int TILE_BYTES = 128 * 128;
     static constexpr int OFF_KV = 0;                              // 2 stages x (K, V)
     static constexpr int OFF_DS = 4 * TILE_BYTES;                 // 2 panels
-    static constexpr int OFF_Q = OFF_DS + 2 * TILE_BYTES;         // ring of (Q, dO)
+    static constexpr int OFF_DQ = OFF_DS + 2 * TILE_BYTES;        // fp32 dQ tile on its way out: 2 panels of 32 columns
+    static constexpr int OFF_Q = OFF_DQ + 2 * TILE_BYTES;         // ring of (Q, dO)
     static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (-lse2[128], -delta[128], mq[128])
     static constexpr int ROW_BYTES = 3 * 128 * 4;
     static constexpr int OFF_BAR = OFF_ROW + NSQ * ROW_BYTES;
@@ -508,7 +509,7 @@ struct BwdWalk {
 __global__ void __launch_bounds__(512, 1)
 bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
              const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-             const BwdParams P)
+             const __grid_constant__ CUtensorMap tmDQ, const BwdParams P)
 {
     using C = Bwd64Cfg;
     constexpr int D = 64, NSQ = C::NSQ, TB = C::TILE_BYTES;
@@ -596,19 +597,46 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const int row0 = P.q_begin + wk.qt() * BM;
             const int h = wk.head();
             const bool last = wk.last();
-            ok = __all_sync(0xffffffffu,
-                            mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag));
-            if (!ok)
-                break;
+            ok = mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag);
             tc_fence_after();
-            drain_block(C::TM_DQ + (it & 1) * 64, P.scale,
-                        [&](int i) -> float * {
-                            const int row = row0 + i;
-                            return row < P.q_end
-                                       ? P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D
-                                       : nullptr;
-                        },
-                        B_DQEMPTY + (it & 1));
+            // dQ(it): tensor memory -> registers -> swizzled fp32 tile in shared memory -> one
+            // tiled reduce-add per 32-column panel.  Whole 256-byte rows reach L2 together, which
+            // the L2 takes about 1.6 times faster than the same bytes as scattered 32-byte pieces.
+            {
+                const int rw = (warp & 3) * 32 + lane; // row of the tile = tensor-memory lane
+                uint32_t o[2][32];
+                tmem_ld32(tmem + lane_base + C::TM_DQ + (it & 1) * 64, o[0]);
+                tmem_ld32(tmem + lane_base + C::TM_DQ + (it & 1) * 64 + 32, o[1]);
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(BAR(B_DQEMPTY + (it & 1)));
+                if (threadIdx.x == 384)
+                    bulk_wait_group_read<0>(); // the previous tile has left shared memory
+                ok = bar_and(3, 128, ok);      // the four warps go on, or leave, together
+                if (!ok)
+                    break;
+#pragma unroll
+                for (int pn = 0; pn < 2; ++pn) {
+                    uint8_t *dst = sp + C::OFF_DQ + pn * TB + rw * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        float4 v;
+                        v.x = __uint_as_float(o[pn][4 * c]) * P.scale;
+                        v.y = __uint_as_float(o[pn][4 * c + 1]) * P.scale;
+                        v.z = __uint_as_float(o[pn][4 * c + 2]) * P.scale;
+                        v.w = __uint_as_float(o[pn][4 * c + 3]) * P.scale;
+                        *reinterpret_cast<float4 *>(dst + ((c ^ (rw & 7)) << 4)) = v;
+                    }
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync 3, 128;" ::: "memory");
+                if (threadIdx.x == 384) {
+                    // rows past the partition's end are clipped by the tensor map
+                    tma_reduce_add_3d(&tmDQ, sb + C::OFF_DQ, 0, h, row0 - P.q_begin);
+                    tma_reduce_add_3d(&tmDQ, sb + C::OFF_DQ + TB, 32, h, row0 - P.q_begin);
+                    bulk_commit_group();
+                }
+            }
             if (last) {
                 // every MMA of the work item is complete (the barrier above covers them all)
                 const int g = wk.g;
@@ -629,6 +657,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
             wk.next();
         }
+        if (threadIdx.x == 384)
+            bulk_wait_group<0>();
     } else if (warp >= 8) {
         reg_dec<56>();
         if (warp == 9) {
@@ -1009,6 +1039,18 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         return PEAGLE_ERR_CUDA;
     const int q_len = p.q_end - p.q_begin;
     const int q_pad = p.n_qt * BM;
+    // fp32 dQ staging [q_len][Hq][D] as a tensor for tiled reduce-adds: 32 columns x 128 rows
+    CUtensorMap tmDQ;
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)a.Hq, (cuuint64_t)q_len};
+        cuuint64_t strides[2] = {(cuuint64_t)D * 4, (cuuint64_t)a.Hq * D * 4};
+        cuuint32_t box[3] = {32, 1, 128};
+        cuuint32_t estr[3] = {1, 1, 1};
+        if (enc(&tmDQ, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, a.dq_acc, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return PEAGLE_ERR_CUDA;
+    }
     const size_t n_prep = (size_t)q_len * a.Hq * (D / 8);
     const size_t n_prep_pad = (size_t)q_pad * a.Hq * (D / 8);
     bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
@@ -1051,7 +1093,7 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         if (ev0)
             cudaEventRecord(ev0, s);
         if (D == 64)
-            bwd64_kernel<<<n_sm, 512, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+            bwd64_kernel<<<n_sm, 512, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, tmDQ, P);
         else
             bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
         if (ev1)

@@ -358,11 +358,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     const int st = i % NS, ph = (i / NS) & 1;
                     const int t = P.stok[((size_t)qt * MAX_SINGLE + i) * BM + r];
                     const int col = t - P.sbase[qt * MAX_SINGLE + i];
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
-                                                     mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
-                    if (!ok)
-                        break;
-                    if (t >= 0 && row_ok) {
+                    ok = mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
+                         mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
+                    if (ok && t >= 0 && row_ok) {
                         const uint8_t *krow = sp + C::OFF_K + st * C::TILE_BYTES + col * 128;
                         const uint8_t *vrow = sp + C::OFF_V + st * C::TILE_BYTES + col * 128;
                         float acc = 0.f;
@@ -400,8 +398,11 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                             }
                         }
                     }
-                    // every thread of this tile's four warps is done with the stage
-                    asm volatile("bar.sync %0, 128;" ::"r"(1 + x) : "memory");
+                    // every thread of this tile's four warps is done with the stage (and the four
+                    // warps leave together if a wait ran out)
+                    ok = bar_and(1 + x, 128, ok);
+                    if (!ok)
+                        break;
                     if (r == 0) {
                         mbar_arrive(BAR(B_KEMPTY + st));
                         mbar_arrive(BAR(B_VEMPTY + st));
