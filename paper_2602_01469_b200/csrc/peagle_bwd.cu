@@ -692,7 +692,10 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const int st = it % NSQ, ph = (it / NSQ) & 1;
                 const int row0 = P.q_begin + wk.qt() * BM;
                 const int h = wk.head();
-                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
+                // the stage is free once dK / dQ of the step two back are done: the barrier of
+                // that step's dQ accumulator (two stages, two accumulators, same parity)
+                static_assert(NSQ == 2, "stage = step parity");
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DQFULL + st), ph ^ 1, abort_flag));
                 if (!ok)
                     break;
                 if (lane == 0) {
@@ -736,13 +739,14 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     mma_ss_lo(tmem + C::TM_DP, kv_k + kv + TBU + k * 2, q_k + q + TBU + k * 2, IDESC_S,
                               k > 0);
             };
-            BwdWalk cur, nxt;
-            cur.init(P, blockIdx.x, gridDim.x);
-            nxt = cur;
-            if (nxt.valid)
-                nxt.next();
+            // The issuing thread is a serial instruction stream, so it keeps its bookkeeping
+            // minimal: per work item only the number of steps (query tiles x heads).
+            const int total = P.counters[1] * P.Hkv;
+            const int G = P.Hq / P.Hkv;
+            int idx = blockIdx.x;
+            int n_cur = idx < total ? P.bitems[idx / P.Hkv].w * G : 0;
             bool ok = true;
-            if (cur.valid) {
+            if (n_cur > 0) {
                 ok = mbar_wait(BAR(B_KVFULL + 0), 0, abort_flag) &&
                      mbar_wait(BAR(B_QFULL + 0), 0, abort_flag);
                 if (ok) {
@@ -753,60 +757,65 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     tc_commit(BAR(B_DPFULL));
                 }
             }
-            for (int it = 0; ok && cur.valid; ++it) {
-                const int st = it % NSQ;
-                const int ks = cur.w & 1;
-                const uint32_t kvo = 2 * ks * TBU, qo = st * 2 * TBU;
-                const bool first = cur.first(), last = cur.last();
-                const int nst = (it + 1) % NSQ, nph = ((it + 1) / NSQ) & 1;
-                const int nks = nxt.valid ? (nxt.w & 1) : 0;
-                const uint32_t nkvo = 2 * nks * TBU, nqo = nst * 2 * TBU;
-                // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
-                ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
-                if (ok && first)
-                    ok = mbar_wait(BAR(B_ACCFREE), (cur.w & 1) ^ 1, abort_flag);
-                if (!ok)
-                    break;
-                tc_fence_after();
-#pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
-                              q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
-                if (nxt.valid) {
-                    if (nxt.first())
-                        ok = mbar_wait(BAR(B_KVFULL + nks), (nxt.w >> 1) & 1, abort_flag);
-                    ok = ok && mbar_wait(BAR(B_QFULL + nst), nph, abort_flag);
+            int it = 0;
+            for (int w = 0; ok && n_cur > 0; ++w) {
+                const int idx_n = idx + (int)gridDim.x;
+                const int n_nxt = idx_n < total ? P.bitems[idx_n / P.Hkv].w * G : 0;
+                const int ks = w & 1, nks_item = (w + 1) & 1;
+                const uint32_t kvo = 2 * ks * TBU;
+                for (int i = 0; ok && i < n_cur; ++i, ++it) {
+                    const int st = it & 1, nst = st ^ 1;
+                    static_assert(NSQ == 2, "stage = step parity");
+                    const uint32_t qo = st * 2 * TBU, nqo = nst * 2 * TBU;
+                    const bool first = i == 0, last = i == n_cur - 1;
+                    const bool has_next = !last || n_nxt > 0;
+                    const uint32_t nkvo = last ? 2 * nks_item * TBU : kvo;
+                    // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
+                    ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
+                    if (ok && first)
+                        ok = mbar_wait(BAR(B_ACCFREE), (w & 1) ^ 1, abort_flag);
                     if (!ok)
                         break;
                     tc_fence_after();
-                    issue_s(nkvo, nqo);
-                    tc_commit(BAR(B_SFULL));
-                }
-                // ---- dK(it), dQ(it) once dS^T(it) is in shared memory, then dP^T(it+1)
-                ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag) &&
-                     mbar_wait(BAR(B_DQEMPTY + (it & 1)), ((it >> 1) & 1) ^ 1, abort_flag);
-                if (!ok)
-                    break;
-                tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    mma_ss_lo(tmem + C::TM_DK, ds_k + (k / 4) * TBU + (k % 4) * 2, q_m + qo + k * 128,
-                              IDESC_KV, !first || k > 0);
+                    for (int k = 0; k < 8; ++k)
+                        mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                                  q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
+                    if (has_next) {
+                        if (last)
+                            ok = mbar_wait(BAR(B_KVFULL + nks_item), ((w + 1) >> 1) & 1, abort_flag);
+                        ok = ok && mbar_wait(BAR(B_QFULL + nst), ((it + 1) >> 1) & 1, abort_flag);
+                        if (!ok)
+                            break;
+                        tc_fence_after();
+                        issue_s(nkvo, nqo);
+                        tc_commit(BAR(B_SFULL));
+                    }
+                    // ---- dK(it), dQ(it) once dS^T(it) is in shared memory, then dP^T(it+1)
+                    ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag) &&
+                         mbar_wait(BAR(B_DQEMPTY + st), ((it >> 1) & 1) ^ 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    mma_ss_lo(tmem + C::TM_DQ + (it & 1) * 64, ds_m + k * 128, kv_m + kvo + k * 128,
-                              IDESC_DQ, k > 0);
-                tc_commit(BAR(B_DQFULL + (it & 1)));
-                tc_commit(BAR(B_QEMPTY + st));
-                if (last)
-                    tc_commit(BAR(B_KVEMPTY + ks));
-                if (nxt.valid) {
-                    issue_dp(nkvo, nqo);
-                    tc_commit(BAR(B_DPFULL));
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss_lo(tmem + C::TM_DK, ds_k + (k / 4) * TBU + (k % 4) * 2,
+                                  q_m + qo + k * 128, IDESC_KV, !first || k > 0);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        mma_ss_lo(tmem + C::TM_DQ + st * 64, ds_m + k * 128, kv_m + kvo + k * 128,
+                                  IDESC_DQ, k > 0);
+                    // also releases the (Q, dO) stage of this step: same parity as the dQ buffer
+                    tc_commit(BAR(B_DQFULL + st));
+                    if (last)
+                        tc_commit(BAR(B_KVEMPTY + ks));
+                    if (has_next) {
+                        issue_dp(nkvo, nqo);
+                        tc_commit(BAR(B_DPFULL));
+                    }
                 }
-                cur = nxt;
-                if (nxt.valid)
-                    nxt.next();
+                idx = idx_n;
+                n_cur = n_nxt;
             }
         }
     } else {
