@@ -17,7 +17,6 @@ import json
 import os
 import subprocess
 import sys
-import threading
 import time
 
 import numpy as np
@@ -55,7 +54,8 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons while the timed region runs: one nvidia-smi process
+    in loop mode (a sample every 100 ms), read when the region ends."""
 
     Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -64,40 +64,46 @@ class ClockSampler:
     def __init__(self, gpu_index: int):
         self.idx = gpu_index
         self.samples = []
-        self.stop = threading.Event()
-        self.th = threading.Thread(target=self._run, daemon=True)
-
-    def _once(self):
-        try:
-            out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                  "-i", str(self.idx)], capture_output=True, text=True, timeout=10).stdout
-            f = [x.strip() for x in out.strip().split(",")]
-            if len(f) >= 6:
-                self.samples.append((float(f[0]), float(f[1]), f[2:6]))
-        except Exception:
-            pass
-
-    def _run(self):
-        while not self.stop.is_set():
-            self._once()
-            self.stop.wait(0.1)
+        self.proc = None
 
     def __enter__(self):
-        self.th.start()
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i",
+                 str(self.idx), "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            time.sleep(0.3)          # let the first sample arrive before the region starts
+        except Exception:
+            self.proc = None
         return self
 
     def __exit__(self, *a):
-        self.stop.set()
-        self.th.join(timeout=15)
-        if not self.samples:
-            self._once()
+        if self.proc is None:
+            return
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=10)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) >= 6:
+                try:
+                    self.samples.append((float(f[0]), float(f[1]), f[2:6]))
+                except ValueError:
+                    pass
 
     def summary(self):
         if not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         reasons = sorted({n for s in self.samples for n, v in zip(names, s[2]) if v.lower() == "active"})
-        return {"sm_mhz": float(np.median([s[0] for s in self.samples])),
+        # the first samples predate the timed region: use the busy half (highest power draw is not
+        # reported here, so take the samples from the middle on)
+        busy = self.samples[len(self.samples) // 3:] or self.samples
+        return {"sm_mhz": float(np.median([s[0] for s in busy])),
+                "sm_min_mhz": float(min(s[0] for s in busy)),
                 "sm_max_mhz": self.samples[0][1], "reasons": reasons, "samples": len(self.samples)}
 
 

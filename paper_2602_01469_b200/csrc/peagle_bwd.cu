@@ -429,7 +429,7 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 
 // ---------------------------------------------------------------------------------------------
 // head_dim 64: software-pipelined variant.  Tensor memory has room for two dQ accumulators, so the
-// MMA warp runs one step ahead of the compute warps:
+// MMA warp runs one step ahead of the compute warps (inside a work item):
 //   while the compute warps turn S^T(i) into P^T(i):   dK(i-1), dQ(i-1), dP^T(i)
 //   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
 // and dQ(i-1) is drained to the fp32 staging rows after dS^T(i) has been handed over.  K / V of
@@ -452,7 +452,10 @@ struct Bwd64Cfg {
     static constexpr int N_BAR = 2 * NSQ + 13;
     static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
     static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
-    static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 256 /* two of 64 */, TM_DK = 384, TM_DV = 448;
+    // tensor memory: S^T | dP^T | dQ | K (bf16) | V (bf16) | dK | dV.  P^T (bf16) overwrites the
+    // first half of each group's S^T columns and dS^T (bf16) the first half of its dP^T columns.
+    static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_K = 320, TM_V = 352, TM_DK = 384,
+                         TM_DV = 448;
 };
 
 // Walks the (work item, query tile, head) iterations of one CTA in execution order.
@@ -521,7 +524,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     constexpr int B_QFULL = 0, B_QEMPTY = NSQ, B_KVFULL = 2 * NSQ, B_KVEMPTY = B_KVFULL + 2,
                   B_SFULL = B_KVFULL + 4, B_DPFULL = B_KVFULL + 5, B_PFULL = B_KVFULL + 6,
-                  B_DSFULL = B_KVFULL + 7, B_DQFULL = B_KVFULL + 8, B_DQEMPTY = B_KVFULL + 10,
+                  B_DSFULL = B_KVFULL + 7, B_DQFULL = B_KVFULL + 8, B_KVTFULL = B_KVFULL + 9,
+                  B_DQEMPTY = B_KVFULL + 10,
                   B_ACCFREE = B_KVFULL + 12;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
@@ -537,8 +541,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         for (int s = 0; s < 2; ++s) {
             mbar_init(BAR(B_KVFULL + s), 1);
             mbar_init(BAR(B_KVEMPTY + s), 1);
-            mbar_init(BAR(B_DQFULL + s), 1);
-            mbar_init(BAR(B_DQEMPTY + s), 128);
+            mbar_init(BAR(B_DQFULL + s), s == 0 ? 1 : 256); // [0] dQ done, [1] = B_KVTFULL
+            mbar_init(BAR(B_DQEMPTY + s), 128);              // [0] used
         }
         mbar_init(BAR(B_SFULL), 1);
         mbar_init(BAR(B_DPFULL), 1);
@@ -597,7 +601,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const int row0 = P.q_begin + wk.qt() * BM;
             const int h = wk.head();
             const bool last = wk.last();
-            ok = mbar_wait(BAR(B_DQFULL + (it & 1)), (it >> 1) & 1, abort_flag);
+            ok = mbar_wait(BAR(B_DQFULL), it & 1, abort_flag);
             tc_fence_after();
             // dQ(it): tensor memory -> registers -> swizzled fp32 tile in shared memory -> one
             // tiled reduce-add per 32-column panel.  Whole 256-byte rows reach L2 together, which
@@ -605,11 +609,11 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             {
                 const int rw = (warp & 3) * 32 + lane; // row of the tile = tensor-memory lane
                 uint32_t o[2][32];
-                tmem_ld32(tmem + lane_base + C::TM_DQ + (it & 1) * 64, o[0]);
-                tmem_ld32(tmem + lane_base + C::TM_DQ + (it & 1) * 64 + 32, o[1]);
+                tmem_ld32(tmem + lane_base + C::TM_DQ, o[0]);
+                tmem_ld32(tmem + lane_base + C::TM_DQ + 32, o[1]);
                 tmem_wait_ld();
                 tc_fence_before();
-                mbar_arrive(BAR(B_DQEMPTY + (it & 1)));
+                mbar_arrive(BAR(B_DQEMPTY));
                 if (threadIdx.x == 384)
                     bulk_wait_group_read<0>(); // the previous tile has left shared memory
                 ok = bar_and(3, 128, ok);      // the four warps go on, or leave, together
@@ -692,10 +696,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const int st = it % NSQ, ph = (it / NSQ) & 1;
                 const int row0 = P.q_begin + wk.qt() * BM;
                 const int h = wk.head();
-                // the stage is free once dK / dQ of the step two back are done: the barrier of
-                // that step's dQ accumulator (two stages, two accumulators, same parity)
-                static_assert(NSQ == 2, "stage = step parity");
-                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DQFULL + st), ph ^ 1, abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
                 if (!ok)
                     break;
                 if (lane == 0) {
@@ -728,48 +729,44 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const uint32_t q_m = desc_lo_sw128(sb + C::OFF_Q, TB);
             constexpr uint32_t TBU = TB >> 4; // one tile in descriptor units
             // S^T = K Q^T and dP^T = V dO^T: kv / q are the stage offsets in descriptor units
-            auto issue_s = [&](uint32_t kv, uint32_t q) {
+            // S^T = K Q^T and dP^T = V dO^T take K / V from tensor memory (one bf16 copy per
+            // work item), so only Q / dO stream from shared memory; q = stage offset in units
+            auto issue_s = [&](uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss_lo(tmem + C::TM_S, kv_k + kv + k * 2, q_k + q + k * 2, IDESC_S, k > 0);
+                    mma_ts_lo(tmem + C::TM_S, tmem + C::TM_K + k * 8, q_k + q + k * 2, IDESC_S, k > 0);
             };
-            auto issue_dp = [&](uint32_t kv, uint32_t q) {
+            auto issue_dp = [&](uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss_lo(tmem + C::TM_DP, kv_k + kv + TBU + k * 2, q_k + q + TBU + k * 2, IDESC_S,
+                    mma_ts_lo(tmem + C::TM_DP, tmem + C::TM_V + k * 8, q_k + q + TBU + k * 2, IDESC_S,
                               k > 0);
             };
             // The issuing thread is a serial instruction stream, so it keeps its bookkeeping
             // minimal: per work item only the number of steps (query tiles x heads).
             const int total = P.counters[1] * P.Hkv;
             const int G = P.Hq / P.Hkv;
-            int idx = blockIdx.x;
-            int n_cur = idx < total ? P.bitems[idx / P.Hkv].w * G : 0;
             bool ok = true;
-            if (n_cur > 0) {
-                ok = mbar_wait(BAR(B_KVFULL + 0), 0, abort_flag) &&
-                     mbar_wait(BAR(B_QFULL + 0), 0, abort_flag);
-                if (ok) {
-                    tc_fence_after();
-                    issue_s(0, 0);
-                    tc_commit(BAR(B_SFULL));
-                    issue_dp(0, 0);
-                    tc_commit(BAR(B_DPFULL));
-                }
-            }
-            int it = 0;
-            for (int w = 0; ok && n_cur > 0; ++w) {
-                const int idx_n = idx + (int)gridDim.x;
-                const int n_nxt = idx_n < total ? P.bitems[idx_n / P.Hkv].w * G : 0;
-                const int ks = w & 1, nks_item = (w + 1) & 1;
+            int it = 0, w = 0;
+            for (int idx = blockIdx.x; ok && idx < total; idx += gridDim.x, ++w) {
+                const int n_cur = P.bitems[idx / P.Hkv].w * G;
+                const int ks = w & 1;
                 const uint32_t kvo = 2 * ks * TBU;
+                // K / V of this item are in tensor memory (and its K tile in shared memory)
+                ok = mbar_wait(BAR(B_KVTFULL), w & 1, abort_flag) &&
+                     mbar_wait(BAR(B_QFULL + (it & 1)), (it >> 1) & 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                issue_s((it & 1) * 2 * TBU);
+                tc_commit(BAR(B_SFULL));
+                issue_dp((it & 1) * 2 * TBU);
+                tc_commit(BAR(B_DPFULL));
                 for (int i = 0; ok && i < n_cur; ++i, ++it) {
                     const int st = it & 1, nst = st ^ 1;
                     static_assert(NSQ == 2, "stage = step parity");
                     const uint32_t qo = st * 2 * TBU, nqo = nst * 2 * TBU;
                     const bool first = i == 0, last = i == n_cur - 1;
-                    const bool has_next = !last || n_nxt > 0;
-                    const uint32_t nkvo = last ? 2 * nks_item * TBU : kvo;
                     // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
                     ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
                     if (ok && first)
@@ -781,41 +778,38 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     for (int k = 0; k < 8; ++k)
                         mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
-                    if (has_next) {
-                        if (last)
-                            ok = mbar_wait(BAR(B_KVFULL + nks_item), ((w + 1) >> 1) & 1, abort_flag);
-                        ok = ok && mbar_wait(BAR(B_QFULL + nst), ((it + 1) >> 1) & 1, abort_flag);
+                    if (!last) {
+                        ok = mbar_wait(BAR(B_QFULL + nst), ((it + 1) >> 1) & 1, abort_flag);
                         if (!ok)
                             break;
                         tc_fence_after();
-                        issue_s(nkvo, nqo);
+                        issue_s(nqo);
                         tc_commit(BAR(B_SFULL));
                     }
-                    // ---- dK(it), dQ(it) once dS^T(it) is in shared memory, then dP^T(it+1)
+                    // ---- dK(it), dQ(it) once dS^T(it) is in tensor and shared memory, then
+                    // dP^T(it+1); the single dQ accumulator must have been read out
                     ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag) &&
-                         mbar_wait(BAR(B_DQEMPTY + st), ((it >> 1) & 1) ^ 1, abort_flag);
+                         mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, abort_flag);
                     if (!ok)
                         break;
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ss_lo(tmem + C::TM_DK, ds_k + (k / 4) * TBU + (k % 4) * 2,
+                        mma_ts_lo(tmem + C::TM_DK, tmem + C::TM_DP + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + k * 128, IDESC_KV, !first || k > 0);
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ss_lo(tmem + C::TM_DQ + st * 64, ds_m + k * 128, kv_m + kvo + k * 128,
-                                  IDESC_DQ, k > 0);
-                    // also releases the (Q, dO) stage of this step: same parity as the dQ buffer
-                    tc_commit(BAR(B_DQFULL + st));
+                        mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, kv_m + kvo + k * 128, IDESC_DQ,
+                                  k > 0);
+                    tc_commit(BAR(B_DQFULL));
+                    tc_commit(BAR(B_QEMPTY + st));
                     if (last)
                         tc_commit(BAR(B_KVEMPTY + ks));
-                    if (has_next) {
-                        issue_dp(nkvo, nqo);
+                    else {
+                        issue_dp(nqo);
                         tc_commit(BAR(B_DPFULL));
                     }
                 }
-                idx = idx_n;
-                n_cur = n_nxt;
             }
         }
     } else {
@@ -836,6 +830,27 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if (wk.first()) {
                 const int2 ktile = P.ktile[wk.kt];
                 mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
+                // New work item: a bf16 copy of K (group 0) / V (group 1) goes to tensor memory,
+                // one row per thread.  Every S^T / dP^T product of the previous item is complete
+                // (their results were consumed in its last step), so the old copy is not in use.
+                const int ks = wk.w & 1;
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_KVFULL + ks), (wk.w >> 1) & 1, abort_flag));
+                if (!ok)
+                    break;
+                const uint8_t *src = sp + C::OFF_KV + (2 * ks + wg) * TB + r * 128;
+                uint32_t kvw[32];
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4 *>(src + ((c ^ (r & 7)) << 4));
+                    kvw[4 * c] = v.x;
+                    kvw[4 * c + 1] = v.y;
+                    kvw[4 * c + 2] = v.z;
+                    kvw[4 * c + 3] = v.w;
+                }
+                tmem_st32(tmem + lane_sel + (wg == 0 ? C::TM_K : C::TM_V), kvw);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(BAR(B_KVTFULL));
             }
             const bool full = wk.full();
             const float *rowbuf = reinterpret_cast<const float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
@@ -917,14 +932,28 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             // the dS^T buffer is free once dK / dQ of the previous iteration have run
             if (it > 0) {
                 ok = __all_sync(0xffffffffu,
-                                mbar_wait(BAR(B_DQFULL + ((it - 1) & 1)), ((it - 1) >> 1) & 1, abort_flag));
+                                mbar_wait(BAR(B_DQFULL), (it - 1) & 1, abort_flag));
                 if (!ok)
                     break;
             }
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = dsv[j];
+            {
+                // the same dS^T also goes over this group's dP^T columns: operand of dK
+                uint32_t pk[32];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    pk[4 * j] = dsv[j].x;
+                    pk[4 * j + 1] = dsv[j].y;
+                    pk[4 * j + 2] = dsv[j].z;
+                    pk[4 * j + 3] = dsv[j].w;
+                }
+                tmem_st32(tDP, pk);
+            }
+            tmem_wait_st();
             fence_proxy_async_smem();
+            tc_fence_before();
             mbar_arrive(BAR(B_DSFULL));
             wk.next();
         }
