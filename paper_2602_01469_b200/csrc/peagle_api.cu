@@ -114,7 +114,7 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.qorder = c.take<int>(nq);
     const size_t nch = (nq + BWD_CQ - 1) / BWD_CQ;
     p.cmask = c.take<uint16_t>(nch * nk);
-    p.ccount = c.take<int>(nch);
+    p.ccount = c.take<int>(nch * BWD_CQ);
     p.bitems = c.take<int4>(nch * nk);
     p.scount = c.take<int>(nq);
     p.skt = c.take<int>(nq * MAX_SINGLE);

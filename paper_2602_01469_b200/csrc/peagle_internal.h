@@ -46,7 +46,7 @@ struct Plan {
     int *kcount;           // [n_qt]
     int *qorder;           // [n_qt] query tiles, most key tiles first
     uint16_t *cmask;       // [n_ch][n_kt] per chunk of BWD_CQ query tiles: bit b not skipped, bit 8+b FULL
-    int *ccount;           // [n_ch] key tiles with a non-zero word
+    int *ccount;           // [n_ch][BWD_CQ] key tiles whose word has 1, 2, .. BWD_CQ query tiles
     int4 *bitems;          // [n_ch * n_kt] backward work items (key tile, chunk, mask word, query tiles)
     int allow_single;      // 1: the kernels of this head_dim take SINGLE tiles
     int *scount;           // [n_qt] SINGLE tiles found per query tile (may exceed MAX_SINGLE: clamp)

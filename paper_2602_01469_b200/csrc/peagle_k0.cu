@@ -280,16 +280,18 @@ __global__ void k0_schedule(Plan p)
 // group of BWD_CQ consecutive query tiles ("chunk").  Items are laid out chunk-major so that the
 // CTAs running at the same time work on the same few query tiles: their Q / dO rows and their
 // fp32 dQ staging rows then stay in L2.
+// The items with all BWD_CQ query tiles come first, chunk-major; the smaller ones (the chunks on
+// the mask's diagonal) follow in descending size, so that the static round-robin over the CTAs
+// ends on small items and the CTAs finish together.
 // Pass 1, one block per chunk: for every key tile a 16-bit word (bit b: query tile 8c+b is not
-// skipped, bit 8+b: it is FULL), and the number of key tiles with a non-zero word.
+// skipped, bit 8+b: it is FULL), and how many key tiles have 1, 2, .. BWD_CQ query tiles.
 __global__ void k0_chunk_masks(Plan p)
 {
-    __shared__ int total;
+    __shared__ int hist[BWD_CQ];
     const int c = blockIdx.x;
-    if (threadIdx.x == 0)
-        total = 0;
+    if (threadIdx.x < BWD_CQ)
+        hist[threadIdx.x] = 0;
     __syncthreads();
-    int mine = 0;
     for (int kt = threadIdx.x; kt < p.n_kt; kt += blockDim.x) {
         unsigned m = 0;
         for (int b = 0; b < BWD_CQ; ++b) {
@@ -303,58 +305,64 @@ __global__ void k0_chunk_masks(Plan p)
             }
         }
         p.cmask[(size_t)c * p.n_kt + kt] = (uint16_t)m;
-        mine += (m != 0);
+        if (m != 0)
+            atomicAdd(&hist[__popc(m & 0xffu) - 1], 1);
     }
-    for (int o = 16; o > 0; o >>= 1)
-        mine += __shfl_xor_sync(0xffffffffu, mine, o);
-    if ((threadIdx.x & 31) == 0)
-        atomicAdd(&total, mine);
     __syncthreads();
-    if (threadIdx.x == 0)
-        p.ccount[c] = total;
+    if (threadIdx.x < BWD_CQ)
+        p.ccount[c * BWD_CQ + threadIdx.x] = hist[threadIdx.x];
 }
 
-// Pass 2, one block per chunk: items of the chunk, key tiles ascending, behind the items of all
-// earlier chunks.  item = (key tile, chunk, mask word, query tiles in the item).
+// Pass 2, one block per chunk: the items of the chunk go to their size class's region, behind the
+// same-size items of all earlier chunks, key tiles ascending.
+// item = (key tile, chunk, mask word, query tiles in the item).
 __global__ void k0_chunk_items(Plan p)
 {
     __shared__ int warp_cnt[4];
-    __shared__ int base;
-    const int c = blockIdx.x;
-    int before = 0;
-    for (int i = threadIdx.x; i < c; i += blockDim.x)
-        before += p.ccount[i];
-    for (int o = 16; o > 0; o >>= 1)
-        before += __shfl_xor_sync(0xffffffffu, before, o);
-    if (threadIdx.x == 0)
-        base = 0;
-    __syncthreads();
-    if ((threadIdx.x & 31) == 0)
-        atomicAdd(&base, before);
-    __syncthreads();
-    for (int o0 = 0; o0 < p.n_kt; o0 += blockDim.x) {
-        const int kt = o0 + threadIdx.x;
-        unsigned m = 0;
-        if (kt < p.n_kt)
-            m = p.cmask[(size_t)c * p.n_kt + kt];
-        const unsigned bal = __ballot_sync(0xffffffffu, m != 0);
-        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-        if (lane == 0)
-            warp_cnt[wid] = __popc(bal);
-        __syncthreads();
-        int off = base;
-        for (int w = 0; w < wid; ++w)
-            off += warp_cnt[w];
-        off += __popc(bal & ((1u << lane) - 1u));
-        if (m != 0)
-            p.bitems[off] = make_int4(kt, c, (int)m, __popc(m & 0xffu));
-        __syncthreads();
-        if (threadIdx.x == 0)
-            base += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
-        __syncthreads();
+    __shared__ int base[BWD_CQ]; // where this chunk's items of each size start
+    __shared__ int cursor;
+    const int c = blockIdx.x, n_ch = gridDim.x;
+    if (threadIdx.x < BWD_CQ) {
+        // sizes in output order: BWD_CQ, BWD_CQ-1, .., 1
+        const int sz = threadIdx.x; // index = size - 1
+        int off = 0;
+        for (int s2 = BWD_CQ - 1; s2 > sz; --s2)
+            for (int i = 0; i < n_ch; ++i)
+                off += p.ccount[i * BWD_CQ + s2];
+        for (int i = 0; i < c; ++i)
+            off += p.ccount[i * BWD_CQ + sz];
+        base[sz] = off;
+        if (c == n_ch - 1 && sz == 0)
+            p.counters[1] = off + p.ccount[c * BWD_CQ];
     }
-    if (c == (int)gridDim.x - 1 && threadIdx.x == 0)
-        p.counters[1] = base;
+    __syncthreads();
+    for (int sz = BWD_CQ - 1; sz >= 0; --sz) {
+        if (threadIdx.x == 0)
+            cursor = base[sz];
+        __syncthreads();
+        for (int o0 = 0; o0 < p.n_kt; o0 += blockDim.x) {
+            const int kt = o0 + threadIdx.x;
+            unsigned m = 0;
+            if (kt < p.n_kt)
+                m = p.cmask[(size_t)c * p.n_kt + kt];
+            const bool mine = m != 0 && __popc(m & 0xffu) == sz + 1;
+            const unsigned bal = __ballot_sync(0xffffffffu, mine);
+            const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+            if (lane == 0)
+                warp_cnt[wid] = __popc(bal);
+            __syncthreads();
+            int off = cursor;
+            for (int w = 0; w < wid; ++w)
+                off += warp_cnt[w];
+            off += __popc(bal & ((1u << lane) - 1u));
+            if (mine)
+                p.bitems[off] = make_int4(kt, c, (int)m, sz + 1);
+            __syncthreads();
+            if (threadIdx.x == 0)
+                cursor += warp_cnt[0] + warp_cnt[1] + warp_cnt[2] + warp_cnt[3];
+            __syncthreads();
+        }
+    }
 }
 
 // ---- test hook: the mask as the device predicate sees it -----------------------------------
