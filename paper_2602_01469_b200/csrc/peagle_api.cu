@@ -26,6 +26,9 @@ struct peagle_ctx {
     bool timing = false;
     std::vector<cudaEvent_t> ev[2]; // recorded (start, stop) pairs: [0] forward, [1] backward
     size_t ev_used[2] = {0, 0};
+    // host entry point: copy-in / compute / copy-out streams and their hand-over events
+    cudaStream_t hs[3] = {nullptr, nullptr, nullptr};
+    std::vector<cudaEvent_t> hev;
 };
 
 namespace {
@@ -409,6 +412,11 @@ int peagle_destroy(peagle_ctx *ctx)
     for (int k = 0; k < 2; ++k)
         for (cudaEvent_t e : ctx->ev[k])
             cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->hev)
+        cudaEventDestroy(e);
+    for (cudaStream_t st : ctx->hs)
+        if (st)
+            cudaStreamDestroy(st);
     delete ctx;
     return PEAGLE_OK;
 }
@@ -681,25 +689,97 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
     uint8_t *dLSE = b;            b += up(nlse);
     uint8_t *danchor = b;         b += up(nmeta);
     uint8_t *ddepth = b;
-    CK(cudaMemcpyAsync(dQin, Q, nq, cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(dKin, K, nkv, cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(dVin, V, nkv, cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(ddO, dO, nq, cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(danchor, prob->anchor, nmeta, cudaMemcpyHostToDevice, s));
-    CK(cudaMemcpyAsync(ddepth, prob->depth, nmeta, cudaMemcpyHostToDevice, s));
+    if (T == 0)
+        return PEAGLE_OK;
+    // Three streams: rows of Q / dO go in, partitions are computed, rows of O / LSE / dQ come
+    // back, each query range cut into slices of HOST_SLICE rows so that the copies of one slice
+    // overlap the arithmetic of another (the slices are query partitions like any other: K / V
+    // and the dK / dV accumulators are shared, exactly Section 3.2's within-sequence scheme).
+    {
+        Call tmp;
+        for (int i = 0; i < nparts; ++i) {
+            rc = validate_partition(prob, &parts[i], tmp);
+            if (rc != PEAGLE_OK)
+                return rc;
+        }
+    }
+    for (cudaStream_t &st : ctx->hs)
+        if (!st)
+            CK(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+    cudaStream_t s_in = ctx->hs[0], s_c = ctx->hs[1], s_out = ctx->hs[2];
+    size_t ev_next = 0;
+    auto event = [&]() -> cudaEvent_t {
+        if (ev_next == ctx->hev.size()) {
+            cudaEvent_t e = nullptr;
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess)
+                return nullptr;
+            ctx->hev.push_back(e);
+        }
+        return ctx->hev[ev_next++];
+    };
+    const size_t row_q = (size_t)prob->n_q_heads * prob->head_dim * 2; // bytes of one Q / O row
+    const size_t n_kv = T * prob->n_kv_heads * prob->head_dim;
+    rc = ensure(ctx, ctx->acc_buf, 2 * n_kv * sizeof(float), s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    float *dK_acc = static_cast<float *>(ctx->acc_buf.ptr), *dV_acc = dK_acc + n_kv;
+    CK(cudaMemcpyAsync(dKin, K, nkv, cudaMemcpyHostToDevice, s_in));
+    CK(cudaMemcpyAsync(dVin, V, nkv, cudaMemcpyHostToDevice, s_in));
+    CK(cudaMemcpyAsync(danchor, prob->anchor, nmeta, cudaMemcpyHostToDevice, s_in));
+    CK(cudaMemcpyAsync(ddepth, prob->depth, nmeta, cudaMemcpyHostToDevice, s_in));
+    CK(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s_c));
     peagle_problem_t dprob = *prob;
     dprob.anchor = reinterpret_cast<const int32_t *>(danchor);
     dprob.depth = reinterpret_cast<const int32_t *>(ddepth);
-    rc = peagle_attn_partitioned(ctx, &dprob, parts, nparts, dQin, dKin, dVin, ddO, dOout,
-                                 reinterpret_cast<float *>(dLSE), ddQ, ddK, ddV, s);
-    if (rc != PEAGLE_OK)
-        return rc;
-    CK(cudaMemcpyAsync(O, dOout, nq, cudaMemcpyDeviceToHost, s));
-    CK(cudaMemcpyAsync(LSE, dLSE, nlse, cudaMemcpyDeviceToHost, s));
-    CK(cudaMemcpyAsync(dQ, ddQ, nq, cudaMemcpyDeviceToHost, s));
-    CK(cudaMemcpyAsync(dK, ddK, nkv, cudaMemcpyDeviceToHost, s));
-    CK(cudaMemcpyAsync(dV, ddV, nkv, cudaMemcpyDeviceToHost, s));
-    CK(cudaStreamSynchronize(s));
+    constexpr int HOST_SLICE = 32 * BM;
+    for (int i = 0; i < nparts; ++i) {
+        for (int b0 = parts[i].q.begin; b0 < parts[i].q.end; b0 += HOST_SLICE) {
+            const int b1 = b0 + HOST_SLICE < parts[i].q.end ? b0 + HOST_SLICE : parts[i].q.end;
+            const size_t off = (size_t)b0 * row_q, len = (size_t)(b1 - b0) * row_q;
+            peagle_partition_t sl = parts[i];
+            sl.q.begin = b0;
+            sl.q.end = b1;
+            CK(cudaMemcpyAsync(dQin + off, static_cast<const uint8_t *>(Q) + off, len,
+                               cudaMemcpyHostToDevice, s_in));
+            CK(cudaMemcpyAsync(ddO + off, static_cast<const uint8_t *>(dO) + off, len,
+                               cudaMemcpyHostToDevice, s_in));
+            cudaEvent_t e_in = event(), e_c = event();
+            if (!e_in || !e_c)
+                return PEAGLE_ERR_CUDA;
+            CK(cudaEventRecord(e_in, s_in));
+            CK(cudaStreamWaitEvent(s_c, e_in, 0));
+            Call c;
+            rc = plan_call(ctx, &dprob, &sl, true, s_c, c);
+            if (rc == PEAGLE_OK)
+                rc = run_fwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, reinterpret_cast<float *>(dLSE), s_c);
+            if (rc == PEAGLE_OK)
+                rc = run_bwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, ddO,
+                             reinterpret_cast<float *>(dLSE), ddQ, dK_acc, dV_acc, s_c);
+            if (rc != PEAGLE_OK) {
+                cudaDeviceSynchronize();
+                return rc;
+            }
+            CK(cudaEventRecord(e_c, s_c));
+            CK(cudaStreamWaitEvent(s_out, e_c, 0));
+            CK(cudaMemcpyAsync(static_cast<uint8_t *>(O) + off, dOout + off, len, cudaMemcpyDeviceToHost, s_out));
+            CK(cudaMemcpyAsync(static_cast<uint8_t *>(dQ) + off, ddQ + off, len, cudaMemcpyDeviceToHost, s_out));
+            CK(cudaMemcpy2DAsync(LSE + b0, T * 4, reinterpret_cast<float *>(dLSE) + b0, T * 4,
+                                 (size_t)(b1 - b0) * 4, (size_t)prob->n_q_heads,
+                                 cudaMemcpyDeviceToHost, s_out));
+        }
+    }
+    ctx->launches += launch_cast_grads(dK_acc, dV_acc, ddK, ddV, n_kv, s_c);
+    CK(cudaGetLastError());
+    cudaEvent_t e_done = event();
+    if (!e_done)
+        return PEAGLE_ERR_CUDA;
+    CK(cudaEventRecord(e_done, s_c));
+    CK(cudaStreamWaitEvent(s_out, e_done, 0));
+    CK(cudaMemcpyAsync(dK, ddK, nkv, cudaMemcpyDeviceToHost, s_out));
+    CK(cudaMemcpyAsync(dV, ddV, nkv, cudaMemcpyDeviceToHost, s_out));
+    CK(cudaStreamSynchronize(s_in));
+    CK(cudaStreamSynchronize(s_c));
+    CK(cudaStreamSynchronize(s_out));
     return PEAGLE_OK;
 }
 
