@@ -58,6 +58,10 @@ SMALL = [
     inputs.Workload("two_seqs", (140, 70), 3, 2, 1, 64, n_segments=2, seed=7),
     inputs.Workload("d128_segments", (260,), 4, 8, 2, 128, n_segments=2, seed=8),
     inputs.Workload("many_tiles", (1100,), 2, 8, 1, 64, seed=13),        # > BWD_CQ query tiles per key tile
+    # 20 depths: the deepest query tiles have more one-key-per-row chain tiles than the kernels
+    # take pair by pair, the rest goes through the tensor-core path; 150 anchors: chain tiles
+    # straddle two key tiles
+    inputs.Workload("deep_chains", (150,), 20, 2, 1, 64, seed=14),
 ]
 
 
