@@ -503,8 +503,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     const int c0 = 2 * i + 64 * c; // columns c0, c0+1 of this row
                     const float p0 = fast_exp2(fmaf(__uint_as_float(xr[c0 >> 5][c0 & 31]),
                                                     P.scale_log2, neg_m));
-                    const float p1 = fast_exp2(fmaf(__uint_as_float(xr[(c0 + 1) >> 5][(c0 + 1) & 31]),
-                                                    P.scale_log2, neg_m));
+                    // every fourth exponential goes to the FMA pipe: the two softmax groups
+                    // together would otherwise keep the exp2 unit busy for 2,048 clocks a step
+                    // (a larger share makes instruction issue the limit instead)
+                    const float a1 = fmaf(__uint_as_float(xr[(c0 + 1) >> 5][(c0 + 1) & 31]),
+                                          P.scale_log2, neg_m);
+                    const float p1 = (i & 1) ? exp2_fma(a1) : fast_exp2(a1);
                     sum += p0 + p1;
                     pk[i] = pack_bf16x2(p0, p1);
                 }
