@@ -454,12 +454,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         if (!allowed_packed(mq, mk.w)) xr[c][i + 3] = 0xff800000u;
                     }
             }
-            float mx = -CUDART_INF_F;
+            float mx4[4]; // four independent chains of three-input maxima
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 4; ++c) {
+                mx4[c] = -CUDART_INF_F;
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    mx = fmaxf(mx, __uint_as_float(xr[c][i]));
+                for (int i = 0; i < 32; i += 2)
+                    mx4[c] = max3(mx4[c], __uint_as_float(xr[c][i]), __uint_as_float(xr[c][i + 1]));
+            }
+            float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             mx *= P.scale_log2; // scale > 0, so the max commutes with the scaling
             const float m_new = fmaxf(m, mx);
             if (j == 0 && n_single == 0) {

@@ -391,6 +391,13 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
+
 // 2^x on the FMA pipe, for taking load off the exp2 unit (16 results per clock per SM): round x
 // to the nearest integer n with the 1.5 * 2^23 trick, a cubic for 2^(x - n) on [-0.5, 0.5]
 // (relative error < 8e-5, far below the bf16 rounding the probabilities get anyway), n added to
