@@ -11,7 +11,7 @@ namespace peagle {
 constexpr int BM = 128;          // query rows per tile
 constexpr int BN = 128;          // keys per tile
 constexpr int MAX_KRANGES = 32;  // visible key ranges per partition
-constexpr int BWD_CQ = 8;        // query tiles per backward work item (aligned chunk; at most 8)
+constexpr int BWD_CQ = 4;        // query tiles per backward work item (aligned chunk; at most 8)
 constexpr int32_t META_NONE_Q = -1;         // packed metadata of a row outside the partition (sees nothing)
 constexpr int32_t META_NONE_K = 0x7fffffff; // packed metadata of a key outside the batch (seen by nobody)
 
