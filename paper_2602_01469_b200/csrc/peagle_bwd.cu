@@ -30,6 +30,7 @@ struct BwdParams {
     const int2 *ktile;
     const int4 *bitems;
     const int *counters;
+    int *cursor; // device counter, zero at launch: next (work item, KV head) index to hand out
     const int32_t *meta;
     int *status;
     int n_qt, q_begin, q_end, T;
@@ -449,26 +450,51 @@ struct Bwd64Cfg {
     static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (-lse2[128], -delta[128], mq[128])
     static constexpr int ROW_BYTES = 3 * 128 * 4;
     static constexpr int OFF_BAR = OFF_ROW + NSQ * ROW_BYTES;
-    static constexpr int N_BAR = 2 * NSQ + 13;
-    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
-    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
+    static constexpr int N_BAR = 2 * NSQ + 13 + 4;  // the last four: work-queue slots
+    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8; // tensor-memory base, abort flag, work queue
+    static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;
     // tensor memory: S^T | dP^T | dQ | K (bf16) | V (bf16) | dK | dV.  P^T (bf16) overwrites the
     // first half of each group's S^T columns and dS^T (bf16) the first half of its dP^T columns.
     static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_K = 320, TM_V = 352, TM_DK = 384,
                          TM_DV = 448;
 };
 
-// Walks the (work item, query tile, head) iterations of one CTA in execution order.
+// Walks the (work item, query tile, head) iterations of one CTA in execution order.  Work items
+// are handed out dynamically: the producer warp takes the next (item, KV head) index from a global
+// cursor and publishes it in a four-slot queue in shared memory; the other roles read it there.
+// A CTA that falls behind therefore takes fewer items, and the CTAs running at any time work on a
+// contiguous window of the chunk-major item list (their shared Q / dO rows and dQ staging rows
+// stay in L2), instead of drifting apart as with a static round-robin.
 struct BwdWalk {
     const int4 *bitems;
-    int idx, stride, total, Hkv, G;
+    int *cursor;
+    volatile int *wq;
+    volatile int *abort;
+    uint32_t wqbar;
+    int idx, total, Hkv, G, lane;
+    bool fetcher;
     int kt, g, c, w;
     unsigned mask, em;
     int hh;
     bool valid;
     __device__ void load()
     {
-        valid = idx < total;
+        const int slot = w & 3;
+        if (fetcher) { // the whole producer warp, convergent
+            int v = 0;
+            if (lane == 0)
+                v = atomicAdd(cursor, 1);
+            v = __shfl_sync(0xffffffffu, v, 0);
+            idx = v < total ? v : -1;
+            if (lane == 0) {
+                wq[slot] = idx;
+                sm100::mbar_arrive(wqbar + 8u * slot);
+            }
+        } else {
+            // slot w & 3 was last used four items ago; no role is more than two items behind
+            idx = sm100::mbar_wait(wqbar + 8u * slot, (w >> 2) & 1, abort) ? wq[slot] : -1;
+        }
+        valid = idx >= 0;
         if (!valid)
             return;
         const int4 item = bitems[idx / Hkv];
@@ -479,11 +505,16 @@ struct BwdWalk {
         em = mask & 0xffu;
         hh = 0;
     }
-    __device__ void init(const BwdParams &P, int first, int step)
+    __device__ void init(const BwdParams &P, volatile int *queue, uint32_t queue_bar,
+                         volatile int *abort_flag, bool is_fetcher, int lane_id)
     {
         bitems = P.bitems;
-        idx = first;
-        stride = step;
+        cursor = P.cursor;
+        wq = queue;
+        wqbar = queue_bar;
+        abort = abort_flag;
+        fetcher = is_fetcher;
+        lane = lane_id;
         Hkv = P.Hkv;
         G = P.Hq / P.Hkv;
         total = P.counters[1] * P.Hkv;
@@ -501,7 +532,6 @@ struct BwdWalk {
             hh = 0;
             em &= em - 1;
             if (em == 0) {
-                idx += stride;
                 ++w;
                 load();
             }
@@ -529,6 +559,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                   B_ACCFREE = B_KVFULL + 12;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
+    volatile int *wq = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 16);
+    constexpr int B_WQ = 2 * NSQ + 13;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -538,6 +570,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             mbar_init(BAR(B_QFULL + s), 1);
             mbar_init(BAR(B_QEMPTY + s), 1);
         }
+        for (int s = 0; s < 4; ++s)
+            mbar_init(BAR(B_WQ + s), 1);
         for (int s = 0; s < 2; ++s) {
             mbar_init(BAR(B_KVFULL + s), 1);
             mbar_init(BAR(B_KVEMPTY + s), 1);
@@ -566,7 +600,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sub = lane >> 2, cq = 2 * (lane & 3); // row inside a 16-lane load, first column
         BwdWalk wk;
-        wk.init(P, blockIdx.x, gridDim.x);
+        wk.init(P, wq, BAR(B_WQ), abort_flag, false, lane);
         int2 ktile = make_int2(0, 0);
         bool ok = true;
         // adds a [32 lanes x 64 columns] block of tensor memory, scaled, to fp32 rows in global
@@ -674,7 +708,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 tma_prefetch_desc(&tmV);
             }
             BwdWalk wk;
-            wk.init(P, blockIdx.x, gridDim.x);
+            wk.init(P, wq, BAR(B_WQ), abort_flag, true, lane);
             auto load_kv = [&](int w, int kt, int g) -> bool {
                 bool ok = true;
                 if (lane == 0) {
@@ -744,11 +778,16 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             };
             // The issuing thread is a serial instruction stream, so it keeps its bookkeeping
             // minimal: per work item only the number of steps (query tiles x heads).
-            const int total = P.counters[1] * P.Hkv;
             const int G = P.Hq / P.Hkv;
             bool ok = true;
             int it = 0, w = 0;
-            for (int idx = blockIdx.x; ok && idx < total; idx += gridDim.x, ++w) {
+            for (;; ++w) {
+                // next (work item, KV head) index from the producer's queue
+                if (!mbar_wait(BAR(B_WQ + (w & 3)), (w >> 2) & 1, abort_flag))
+                    break;
+                const int idx = wq[w & 3];
+                if (idx < 0)
+                    break;
                 const int n_cur = P.bitems[idx / P.Hkv].w * G;
                 const int ks = w & 1;
                 const uint32_t kvo = 2 * ks * TBU;
@@ -810,6 +849,8 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         tc_commit(BAR(B_DPFULL));
                     }
                 }
+                if (!ok)
+                    break;
             }
         }
     } else {
@@ -822,7 +863,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const uint32_t tDP = tmem + lane_sel + C::TM_DP + wg * 64;
         uint8_t *dsrow = sp + C::OFF_DS + wg * TB + r * 128;
         BwdWalk wk;
-        wk.init(P, blockIdx.x, gridDim.x);
+        wk.init(P, wq, BAR(B_WQ), abort_flag, false, lane);
         bool ok = true;
         int32_t mk = META_NONE_K;
         for (int it = 0; ok && wk.valid; ++it) {
@@ -1100,6 +1141,7 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         P.ktile = p.ktile;
         P.bitems = p.bitems;
         P.counters = p.counters;
+        P.cursor = p.counters + 2;
         P.meta = p.meta;
         P.status = p.status;
         P.n_qt = p.n_qt;
