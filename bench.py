@@ -28,6 +28,9 @@ from paper_2602_01469_b200 import inputs  # noqa: E402
 
 METRIC = "masked-attn fwd+bwd useful TFLOP/s"
 UNIT = "TFLOP/s"
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (set back to None whenever that kernel changes).
+NCU_TRAFFIC_BYTES = {"gptoss_n4096": 2940853504 + 1447944448}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
@@ -265,8 +268,9 @@ def run_cuda(args, w):
         launches_per_step = max(n_bwd // args.steps, 1)
         achieved = (f_bwd / launches_per_step) / (bwd_ms_launch * 1e-3) / 1e12
         roofline = {
-            "kernel": "bwd_kernel", "bound": "tensor", "achieved": achieved, "peak": peak,
-            "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+            "kernel": "bwd64_kernel" if w.head_dim == 64 else "bwd_kernel<128>", "bound": "tensor",
+            "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+            "traffic": NCU_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch (ncu, DRAM)",
             "peak_source": f"{peak_kind} bf16_tflops (burst)",
             "ms_per_launch": bwd_ms_launch, "launches_timed": int(n_bwd),
             "fwd_kernel": {"achieved": (f_fwd / launches_per_step) / (fwd_ms_launch * 1e-3) / 1e12,
