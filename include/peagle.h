@@ -191,7 +191,7 @@ int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
 /*
  * The same driver with HOST tensors (pinned memory, or the copies do not overlap anything).
  * K, V and the metadata go to the device first; then every partition's query range is cut into
- * slices of 4,096 rows that are themselves run as query partitions (Section 3.2's scheme: K / V
+ * slices of 2,048 rows that are themselves run as query partitions (Section 3.2's scheme: K / V
  * and the fp32 dK / dV sums are shared), so that the copy-in of Q / dO rows, the arithmetic and
  * the copy-out of O / LSE / dQ rows of different slices overlap on three internal streams.  Only
  * rows that belong to a partition are written to O, LSE and dQ.  prob->anchor / prob->depth are

@@ -731,7 +731,7 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
     peagle_problem_t dprob = *prob;
     dprob.anchor = reinterpret_cast<const int32_t *>(danchor);
     dprob.depth = reinterpret_cast<const int32_t *>(ddepth);
-    constexpr int HOST_SLICE = 32 * BM;
+    constexpr int HOST_SLICE = 16 * BM;
     for (int i = 0; i < nparts; ++i) {
         for (int b0 = parts[i].q.begin; b0 < parts[i].q.end; b0 += HOST_SLICE) {
             const int b1 = b0 + HOST_SLICE < parts[i].q.end ? b0 + HOST_SLICE : parts[i].q.end;
