@@ -34,10 +34,19 @@ NCU_TRAFFIC_BYTES = {"gptoss_n4096": 2940853504 + 1447944448}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
+def grid(w: inputs.Workload, i: int, n: int):
+    """Metadata of sequence i of a workload: the full grid, or its COD-subsampled version."""
+    return inputs.full_grid(n, w.K) if w.cod_r is None else inputs.cod_grid(n, w.K, w.cod_r, w.seed + i)
+
+
 def allowed_pairs(w: inputs.Workload) -> int:
-    """Allowed (query, key) pairs of a full-grid workload: a token (anchor a, depth d) sees the
-    a+1 real tokens up to its anchor and its d chain tokens."""
-    return sum(w.K * n * (n + 1) // 2 + n * w.K * (w.K - 1) // 2 for n in w.seq_lens)
+    """Allowed (query, key) pairs: a token (anchor a, depth d) sees the a+1 real tokens up to its
+    anchor and its d chain tokens (all present: the kept sets are nested along chains)."""
+    total = 0
+    for i, n in enumerate(w.seq_lens):
+        a, d = grid(w, i, n)
+        total += int(a.astype(np.int64).sum() + d.astype(np.int64).sum() + a.shape[0])
+    return total
 
 
 def useful_flops(w: inputs.Workload):
@@ -117,9 +126,10 @@ def oracle_sample(w: inputs.Workload, budget_s: float, seed: int = 0):
     from oracle import partition as opart
     from oracle import peagle_oracle as orc
 
-    n = max(w.seq_lens)
-    anchor, depth = inputs.full_grid(n, w.K)
-    T = n * w.K
+    i_long = int(np.argmax(w.seq_lens))
+    n = w.seq_lens[i_long]
+    anchor, depth = grid(w, i_long, n)
+    T = int(anchor.shape[0])
     Q, K, V, dO = inputs.make_tensors(T, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed)
     Qf, Kf, Vf, dOf = (t.float().numpy() for t in (Q, K, V, dO))
     rng = np.random.default_rng(seed)

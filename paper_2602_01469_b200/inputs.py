@@ -26,9 +26,13 @@ class Workload:
     n_segments: int = 1      # segments per sequence (even boundaries), when seg_len is None
     seg_len: int | None = None   # fixed segment length in context tokens (overrides n_segments)
     seed: int = 0
+    cod_r: float | None = None   # COD retention rate (Section 3): depth d keeps about n * r^d chains
 
     @property
     def total_tokens(self) -> int:
+        if self.cod_r is not None:
+            return sum(int(cod_grid(n, self.K, self.cod_r, self.seed + i)[0].shape[0])
+                       for i, n in enumerate(self.seq_lens))
         return sum(self.seq_lens) * self.K
 
     @property
@@ -61,6 +65,8 @@ WORKLOADS = {
                                 seg_len=8192, seed=50),
 }
 # a half-length copy of the headline shape, small enough for profiler captures
+# the paper's own example of Section 3.2: 8,192 tokens, K = 8, retention 0.8 (about 34K positions)
+WORKLOADS["gptoss_n8192_cod"] = Workload("gptoss_n8192_cod", (8192,), 8, 64, 8, 64, seed=60, cod_r=0.8)
 WORKLOADS["gptoss_n2048_profile"] = Workload("gptoss_n2048_profile", (2048,), 8, 64, 8, 64, seed=31)
 HEADLINE = "gptoss_n4096"
 
@@ -70,6 +76,25 @@ def full_grid(n: int, K: int):
     depth = np.repeat(np.arange(K, dtype=np.int32), n)
     anchor = np.tile(np.arange(n, dtype=np.int32), K)
     return anchor, depth
+
+
+def cod_grid(n: int, K: int, r: float, seed: int):
+    """COD down-sampling of the full grid (Section 3: depth 0 keeps all n positions, depth d
+    about n * r^d, drawn at random per example; Section 3.2: position p at depth d needs position
+    p-1 at depth d-1, so the sets are nested along chains).  Depth d keeps round(r * kept(d-1)) of
+    the chains still alive at depth d-1, chosen uniformly with ``numpy.random.default_rng(seed)``;
+    a chain whose position anchor + d would pass the end of the sequence is not continued, as in
+    the printed example.  Returns anchor, depth (depth-major, anchors ascending)."""
+    rng = np.random.default_rng(seed)
+    alive = np.arange(n, dtype=np.int32)
+    anchors, depths = [alive], [np.zeros(n, np.int32)]
+    for d in range(1, K):
+        alive = alive[alive + d < n]
+        keep = min(int(round(r * anchors[-1].shape[0])), alive.shape[0])
+        alive = np.sort(rng.choice(alive, size=keep, replace=False)).astype(np.int32)
+        anchors.append(alive)
+        depths.append(np.full(keep, d, np.int32))
+    return np.concatenate(anchors), np.concatenate(depths)
 
 
 def position_sets(anchor: np.ndarray, depth: np.ndarray, K: int) -> list:
@@ -140,7 +165,7 @@ def build_case(w: Workload, assign_fn):
     cu = [0]
     anchors, depths, parts = [], [], []
     for i, n in enumerate(w.seq_lens):
-        a, d = full_grid(n, w.K)
+        a, d = full_grid(n, w.K) if w.cod_r is None else cod_grid(n, w.K, w.cod_r, w.seed + i)
         bounds = segment_boundaries(n, w.n_segments, w.seg_len)
         if len(bounds) > 2:
             seg = np.asarray(assign_fn(a, d, w.K, bounds), dtype=np.int32)

@@ -43,6 +43,9 @@ SMALL = [
     # take pair by pair, the rest goes through the tensor-core path; 150 anchors: chain tiles
     # straddle two key tiles
     inputs.Workload("deep_chains", (150,), 20, 2, 1, 64, seed=14),
+    # COD-subsampled metadata (retention 0.7): ragged depth blocks, chain tiles that are no
+    # diagonals, Algorithm 1 on nested position sets
+    inputs.Workload("cod_segments", (700,), 6, 4, 2, 64, n_segments=2, seed=15, cod_r=0.7),
 ]
 
 
