@@ -137,7 +137,7 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
  * part of the library image instead.  It calls no cudaMalloc, cudaFree or any routine that
  * allocates.
  *
- * Cost and limits: the array is PEAGLE_STATIC_SCRATCH_BYTES (2 MiB) of device memory on every
+ * Cost and limits: the array is PEAGLE_STATIC_SCRATCH_BYTES (4 MiB) of device memory on every
  * GPU that loads the library, held until the process exits.  Accepted sizes:
  * prob->total_tokens <= PEAGLE_STATIC_MAX_TOKENS and (query tiles of the partition) x (key tiles
  * of its visible ranges) <= PEAGLE_STATIC_MAX_TILE_PAIRS, tiles as peagle_tile_shape reports
@@ -155,7 +155,7 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
  * streams, or different host threads -- race on it: keep them on one stream or order them with
  * events.  Q, K, V, O, LSE, prob and part exactly as for peagle_attn_fwd.
  */
-#define PEAGLE_STATIC_SCRATCH_BYTES (2u << 20)
+#define PEAGLE_STATIC_SCRATCH_BYTES (4u << 20)
 #define PEAGLE_STATIC_MAX_TOKENS 32768
 #define PEAGLE_STATIC_MAX_TILE_PAIRS 65536
 int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,

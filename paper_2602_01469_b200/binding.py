@@ -197,7 +197,7 @@ def peagle_attn_fwd(ctx, prob: Problem, part: Partition, Q, K, V, O, LSE, stream
 def peagle_attn_fwd_static(device: int, prob: Problem, part: Partition, Q, K, V, O, LSE,
                            dev_status=None, stream=None):
     """Forward without any device allocation: the call's tile plan lives in a fixed array inside
-    the library (2 MiB per GPU), so no context is needed.  ``dev_status`` is an optional int32
+    the library (4 MiB per GPU), so no context is needed.  ``dev_status`` is an optional int32
     device tensor that receives a device-side error code."""
     _check(lib().peagle_attn_fwd_static(int(device), prob.ref(), part.ref(), _ptr(Q), _ptr(K),
                                         _ptr(V), _ptr(O), _ptr(LSE), _ptr(dev_status),

@@ -123,7 +123,7 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.skt = c.take<int>(nq * MAX_SINGLE);
     p.sorder = c.take<uint8_t>(nq * MAX_SINGLE);
     p.scol = c.take<uint8_t>(nq * MAX_SINGLE * BM);
-    p.stok = c.take<int32_t>(nq * MAX_SINGLE * BM);
+    p.scs = c.take<uint8_t>(nq * MAX_SINGLE * BM);
     p.sbase = c.take<int>(nq * MAX_SINGLE);
     if (bytes_out)
         *bytes_out = c.off + 256;
@@ -304,7 +304,7 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
 // Lives in the library image: every GPU that loads the library holds these bytes until the
 // process exits.  Layout: the K0 plan (carve_plan) from byte 0, a fallback status word in the
 // last 256 bytes.
-constexpr size_t STATIC_SCRATCH_BYTES = size_t(2) << 20;
+constexpr size_t STATIC_SCRATCH_BYTES = size_t(4) << 20;
 constexpr int STATIC_MAX_TOKENS = 32768;
 constexpr int STATIC_MAX_TILE_PAIRS = 65536;
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];

@@ -37,7 +37,7 @@ struct FwdParams {
     float scale_log2;
     // SINGLE tiles (one allowed key per row), handled pair by pair before the tile loop
     const int *scount;
-    const int32_t *stok; // [n_qt][MAX_SINGLE][BM] key token of entry i for row r, or -1
+    const uint8_t *scs;  // [n_qt][MAX_SINGLE][BM] key column of entry i for row r, or NO_COL
     const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
     const __nv_bfloat16 *Q, *K, *V;
 };
@@ -356,11 +356,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     o[i] = 0.f;
                 for (int i = 0; ok && i < n_single; ++i) {
                     const int st = i % NS, ph = (i / NS) & 1;
-                    const int t = P.stok[((size_t)qt * MAX_SINGLE + i) * BM + r];
-                    const int col = t - P.sbase[qt * MAX_SINGLE + i];
+                    const int col = P.scs[((size_t)qt * MAX_SINGLE + i) * BM + r];
                     ok = mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
                          mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
-                    if (ok && t >= 0 && row_ok) {
+                    if (ok && col != NO_COL && row_ok) {
                         const uint8_t *krow = sp + C::OFF_K + st * C::TILE_BYTES + col * 128;
                         const uint8_t *vrow = sp + C::OFF_V + st * C::TILE_BYTES + col * 128;
                         float acc = 0.f;
@@ -622,7 +621,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     P.two = ((a.Hq / a.Hkv) % 2 == 0) ? 1 : 0;
     P.scale_log2 = a.scale * 1.4426950408889634f;
     P.scount = p.scount;
-    P.stok = p.stok;
+    P.scs = p.scs;
     P.sbase = p.sbase;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);

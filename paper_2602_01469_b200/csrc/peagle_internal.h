@@ -54,8 +54,8 @@ struct Plan {
     uint8_t *sorder;       // [n_qt][MAX_SINGLE] slots by ascending key tile
     uint8_t *scol;         // [n_qt][MAX_SINGLE][BM] per row: the one allowed key column, or NO_COL
     int *sbase;            // [n_qt][MAX_SINGLE] first token of entry i's key tile
-    int32_t *stok;         // [n_qt][MAX_SINGLE][BM] what the kernels read: entry i (slots by ascending
-                           // key tile) of row r is the token index of its key, or -1
+    uint8_t *scs;          // [n_qt][MAX_SINGLE][BM] what the kernels read: entry i (slots by ascending
+                           // key tile) of row r is its key's column in that tile, or NO_COL
     int *status;           // device status word
 };
 

@@ -247,8 +247,7 @@ __global__ void k0_lists(Plan p)
         for (int i = 0; i < ns; ++i) {
             const int slot = p.sorder[self * MAX_SINGLE + i];
             const int col = p.scol[((size_t)self * MAX_SINGLE + slot) * BM + threadIdx.x];
-            p.stok[((size_t)self * MAX_SINGLE + i) * BM + threadIdx.x] =
-                col == NO_COL ? -1 : p.ktile[p.skt[self * MAX_SINGLE + slot]].x + col;
+            p.scs[((size_t)self * MAX_SINGLE + i) * BM + threadIdx.x] = (uint8_t)col;
         }
     }
 }

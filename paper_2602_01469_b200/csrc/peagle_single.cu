@@ -19,7 +19,8 @@ using namespace sm100;
 
 struct SingleParams {
     const int *scount;
-    const int32_t *stok; // [n_qt][MAX_SINGLE][BM]
+    const uint8_t *scs;  // [n_qt][MAX_SINGLE][BM] key column of entry i for row r, or NO_COL
+    const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
     const __nv_bfloat16 *Q, *K, *V, *dO;
     const float *nl2, *nd; // [Hq][q_pad]
     float *dq_acc, *dK_acc, *dV_acc;
@@ -85,7 +86,12 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
         bool any = false;
 #pragma unroll
         for (int i = 0; i < KEYS; ++i) {
-            tok[i] = (i0 + i < ns) ? P.stok[((size_t)qt * MAX_SINGLE + i0 + i) * BM + rr] : -1;
+            tok[i] = -1;
+            if (i0 + i < ns) {
+                const int col = P.scs[((size_t)qt * MAX_SINGLE + i0 + i) * BM + rr];
+                if (col != NO_COL)
+                    tok[i] = P.sbase[qt * MAX_SINGLE + i0 + i] + col;
+            }
             any |= tok[i] >= 0;
         }
         if (!any)
@@ -164,7 +170,8 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
         return 0;
     SingleParams P;
     P.scount = p.scount;
-    P.stok = p.stok;
+    P.scs = p.scs;
+    P.sbase = p.sbase;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);
