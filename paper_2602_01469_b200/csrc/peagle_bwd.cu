@@ -1,21 +1,22 @@
 // K2: backward of one query partition on sm_100a (dQ, and fp32 accumulation of dK / dV).
 //
 // Key-tile-outer formulation.  A work item is one key tile (128 keys) of one KV head together
-// with up to BWD_CQ query tiles of its list; for each of those query tiles the item visits the
-// G query heads of the group.  dK and dV of the key tile stay in tensor memory for the whole item
-// and are added to the caller's fp32 accumulators once at its end; dQ of each visited (query
-// tile, head) is added to an fp32 staging buffer and rounded to bf16 by a last kernel.
+// with the non-skipped query tiles of one aligned chunk of BWD_CQ query tiles; for each of those
+// query tiles the item visits the G query heads of the group (one "step" each).  dK and dV of the
+// key tile stay in tensor memory for the whole item and are added to the caller's fp32
+// accumulators once at its end; dQ of each step is added to an fp32 staging buffer and rounded to
+// bf16 by a last kernel.
 //
 // All score-shaped matrices are held transposed (lanes = keys, columns = query rows) so that the
 // probabilities can feed the dV product straight from tensor memory:
-//   S^T  = K Q^T            both operands from shared memory (K-major)
-//   dP^T = V dO^T           both operands from shared memory (K-major)
+//   S^T  = K Q^T,  dP^T = V dO^T
 //   P^T  = exp2(scale*log2e*S^T - LSE*log2e), masked entries 0;  dS^T = P^T o (dP^T - Delta)
 //   dV  += P^T dO           P^T from tensor memory (bf16, over S^T), dO from shared memory (MN-major)
-//   dK  += dS^T Q           dS^T from shared memory (K-major), Q MN-major
-//   dQ   = dS K             dS^T read as an MN-major A operand, K MN-major
-// Roles: warps 0-7 compute (two groups of 128 threads, one key per thread, each group half of
-// the query columns), warp 8 lane 0 issues the MMAs, warp 9 is the TMA producer.
+//   dK  += dS^T Q           Q MN-major
+//   dQ   = dS K             dS^T read from shared memory as an MN-major A operand, K MN-major
+// Two kernels: bwd_kernel<D> (used for head_dim 128; every operand but P^T from shared memory,
+// one step at a time; warps 0-7 compute, warp 8 lane 0 issues the MMAs, warp 9 produces) and
+// bwd64_kernel (head_dim 64, below).
 #include <math_constants.h>
 
 #include "peagle_internal.h"
@@ -429,16 +430,18 @@ bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 }
 
 // ---------------------------------------------------------------------------------------------
-// head_dim 64: software-pipelined variant.  Tensor memory has room for two dQ accumulators, so the
-// MMA warp runs one step ahead of the compute warps (inside a work item):
+// head_dim 64: software-pipelined variant.  The MMA warp runs one step ahead of the compute warps
+// inside a work item:
 //   while the compute warps turn S^T(i) into P^T(i):   dK(i-1), dQ(i-1), dP^T(i)
 //   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
-// and dQ(i-1) is drained to the fp32 staging rows after dS^T(i) has been handed over.  K / V of
-// the next work item are prefetched into a second stage.  512 threads: warps 0-7 compute, warp 8
-// issues MMAs, warp 9 produces, warps 12-15 drain dQ (and dK / dV at the end of a work item) from
-// tensor memory to the fp32 buffers with global reductions.  The drain has warps of its own
-// because a thread with reductions in flight stalls on its next proxy fence, which the compute
-// warps need once per step for the dS^T hand-over.
+// K and V of the item sit in tensor memory as bf16 (A operands of S^T and dP^T), dS^T goes both
+// over the dP^T columns (A operand of dK) and, swizzled, to shared memory (A operand of dQ).
+// K / V tiles of the next item are prefetched into a second shared-memory stage; the items come
+// from a global cursor through a small queue.  512 threads: warps 0-7 compute, warp 8 issues
+// MMAs, warp 9 produces, warps 12-15 drain dQ (through a swizzled fp32 tile in shared memory and
+// tiled reduce-adds) and, at the end of an item, dK / dV (global reductions from registers).
+// The drain has warps of its own because a thread with reductions in flight stalls on its next
+// proxy fence, which the compute warps need once per step for the dS^T hand-over.
 struct Bwd64Cfg {
     static constexpr int D = 64;
     static constexpr int NSQ = 2;
