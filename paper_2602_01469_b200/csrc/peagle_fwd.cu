@@ -2,19 +2,23 @@
 //
 // One CTA owns one query tile (128 rows) for two query heads of the same KV group (or one head
 // when the group size is odd), so both tiles share the K/V tiles staged in shared memory and the
-// same mask.  Roles:
+// same mask.  Roles (384 threads):
 //   warps 0-3  softmax of tile A (one query row per thread; online softmax in the log2 domain,
 //              log-sum-exp bookkeeping, final normalisation and store)
 //   warps 4-7  softmax of tile B
-//   warp  8    allocates tensor memory; lane 0 issues every tcgen05.mma
+//   warp  8    allocates tensor memory; lane 0 issues the MMAs of tile A
+//   warp  10   lane 0 issues the MMAs of tile B
 //   warp  9    producer: TMA loads of Q once and of the K / V tiles through a ring, plus the
 //              packed metadata of each key tile for the implicit mask
-// Tensor memory (512 columns x 128 lanes, fp32): S_A | S_B (128 columns each; the bf16
-// probabilities overwrite the first 64 columns of their own S), then O_A | O_B (head_dim each).
+// Tensor memory (512 columns x 128 lanes, fp32): S_A | S_B (128 columns each), O_A | O_B
+// (head_dim each) and, for head_dim 64, P_A | P_B (bf16 probabilities, 64 columns each) so that
+// S(j+1) is computed while the softmax of S(j) runs; for head_dim 128 tensor memory is full and
+// the probabilities overwrite the first 64 columns of their own S.
 // S = Q K^T takes both operands from shared memory (K-major, 128-byte swizzle); O += P V takes
-// P from tensor memory and V from shared memory (MN-major).  The MMA thread interleaves the two
-// tiles so that the tensor cores work on one while the other is in its softmax.
-// Only tiles the classifier kept are visited; FULL tiles skip the per-element predicate.
+// P from tensor memory and V from shared memory (MN-major).
+// Only tiles the classifier kept are visited; FULL tiles skip the per-element predicate; SINGLE
+// tiles (one allowed key per row, head_dim 64) pass through the same ring first and are done pair
+// by pair on the CUDA cores, their result seeding the running (m, l, O).
 #include <math_constants.h>
 
 #include "peagle_internal.h"
