@@ -1,15 +1,19 @@
 // K1: forward of one query partition on sm_100a.
 //
-// One CTA owns one query tile (128 rows) for two query heads of the same KV group (or one head
+// A work item is one query tile (128 rows) for two query heads of the same KV group (or one head
 // when the group size is odd), so both tiles share the K/V tiles staged in shared memory and the
-// same mask.  Roles (384 threads):
+// same mask.  The kernel is persistent: one CTA per SM (a kernel that allocates tensor memory gets
+// one resident CTA per SM) draws items from a global counter, longest query tiles first, and its
+// barriers, K / V ring and tensor memory carry on from item to item, so that the loads and the
+// first S product of the next item run under the last softmax and the epilogue of the current
+// one.  Roles (384 threads):
 //   warps 0-3  softmax of tile A (one query row per thread; online softmax in the log2 domain,
 //              log-sum-exp bookkeeping, final normalisation and store)
 //   warps 4-7  softmax of tile B
 //   warp  8    allocates tensor memory; lane 0 issues the MMAs of tile A
 //   warp  10   lane 0 issues the MMAs of tile B
-//   warp  9    producer: TMA loads of Q once and of the K / V tiles through a ring, plus the
-//              packed metadata of each key tile for the implicit mask
+//   warp  9    producer: draws the items; TMA loads of Q per item and of the K / V tiles
+//              through a ring, plus the packed metadata of each key tile for the implicit mask
 // Tensor memory (512 columns x 128 lanes, fp32): S_A | S_B (128 columns each), O_A | O_B
 // (head_dim each) and, for head_dim 64, P_A | P_B (bf16 probabilities, 64 columns each) so that
 // S(j+1) is computed while the softmax of S(j) runs; for head_dim 128 tensor memory is full and
@@ -20,6 +24,8 @@
 // tiles (one allowed key per row, head_dim 64) pass through the same ring first and are done pair
 // by pair on the CUDA cores, their result seeding the running (m, l, O).
 #include <math_constants.h>
+
+#include <algorithm>
 
 #include "peagle_internal.h"
 #include "sm100_ptx.cuh"
@@ -33,6 +39,8 @@ struct FwdParams {
     const int *qorder;
     const int32_t *meta;
     int *status;
+    int *cursor;  // next work item (zero at launch)
+    int n_items;  // query tiles x head blocks
     int n_kt, q_begin, q_end, T;
     __nv_bfloat16 *O;
     float *LSE;
@@ -74,9 +82,9 @@ struct FwdCfg {
     static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
     static constexpr int OFF_META = OFF_V + NS * TILE_BYTES;
     static constexpr int OFF_BAR = OFF_META + NS * BN * 4;
-    static constexpr int N_BAR = 1 + 4 * NS + 8;
-    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
-    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024; // + slack for 1024-byte alignment
+    static constexpr int N_BAR = 1 + 4 * NS + 8 + 9;
+    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8; // tmem slot, abort flag, item queue
+    static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024; // + slack for 1024-byte alignment
     static constexpr int TM_S = 0;      // S_A at 0, S_B at 128
     static constexpr int TM_O = 256;    // O_A at 256, O_B at 256 + D
     // head_dim 64 leaves 128 columns for the bf16 probabilities (64 columns per tile), so the next
@@ -104,23 +112,41 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     // barrier indices
     constexpr int B_QFULL = 0, B_KFULL = 1, B_KEMPTY = 1 + NS, B_VFULL = 1 + 2 * NS,
                   B_VEMPTY = 1 + 3 * NS, B_SFULL = 1 + 4 * NS, B_PFULL = B_SFULL + 2,
-                  B_PVDONE = B_SFULL + 4, B_SREAD = B_SFULL + 6;
+                  B_PVDONE = B_SFULL + 4, B_SREAD = B_SFULL + 6, B_WQFULL = B_SFULL + 8,
+                  B_WQFREE = B_WQFULL + 4, B_QEMPTY = B_WQFREE + 4;
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
+    volatile int *wq = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 8); // 4 slots
     int32_t *smeta = reinterpret_cast<int32_t *>(sp + C::OFF_META);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ntile = P.two ? 2 : 1;
     const int n_hb = P.two ? P.Hq / 2 : P.Hq;
-    const int qt = P.qorder[blockIdx.x / n_hb];
-    const int hb = blockIdx.x % n_hb;
-    const int h0 = P.two ? 2 * hb : hb;
-    const int g = h0 / (P.Hq / P.Hkv);
-    const int row0 = P.q_begin + qt * BM;
-    const int cnt = P.kcount[qt];
-    const int2 *klist = P.klist + (size_t)qt * P.n_kt;
-    // SINGLE tiles exist for head_dim 64 only; their result seeds (m, l, O) before the tile loop
-    const int n_single = (D == 64) ? min(P.scount[qt], MAX_SINGLE) : 0;
+    // Work item w of this CTA = (query tile, head block), handed out by a global counter in the
+    // order of the schedule (query tiles with the most key tiles first).  The producer warp draws
+    // the index and passes it to the other roles through a four-slot queue in shared memory.
+    struct Item {
+        int qt, h0, g, row0, cnt, n_single;
+        const int2 *klist;
+    };
+    auto decode = [&](int idx) {
+        Item it;
+        it.qt = P.qorder[idx / n_hb];
+        const int hb = idx % n_hb;
+        it.h0 = P.two ? 2 * hb : hb;
+        it.g = it.h0 / (P.Hq / P.Hkv);
+        it.row0 = P.q_begin + it.qt * BM;
+        it.cnt = P.kcount[it.qt];
+        it.klist = P.klist + (size_t)it.qt * P.n_kt;
+        // SINGLE tiles exist for head_dim 64 only; their result seeds (m, l, O) of the tile loop
+        it.n_single = (D == 64) ? min(P.scount[it.qt], MAX_SINGLE) : 0;
+        return it;
+    };
+    // Roles other than the producer: index of item w, or -1 at the end (or when a wait ran out).
+    auto take = [&](int w) {
+        const int slot = w & 3;
+        return mbar_wait(BAR(B_WQFULL + slot), (w >> 2) & 1, abort_flag) ? wq[slot] : -1;
+    };
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -137,6 +163,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mbar_init(BAR(B_PVDONE + x), 1);
             mbar_init(BAR(B_SREAD + x), 128);
         }
+        for (int i = 0; i < 4; ++i) {
+            mbar_init(BAR(B_WQFULL + i), 1);
+            mbar_init(BAR(B_WQFREE + i), 4 * ntile); // one arrival per softmax warp
+        }
+        // Q may be overwritten once the MMA threads are done with it and every softmax warp has
+        // read its rows (or has no use for them)
+        mbar_init(BAR(B_QEMPTY), 5 * ntile);
         fence_mbar_init();
     }
     if (warp == 8) {
@@ -153,23 +186,46 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         reg_dec<56>();
     if (warp == 9) {
         // ------------------------------------------------------------ producer
-        if (cnt > 0 || n_single > 0) {
-            if (lane == 0) {
-                tma_prefetch_desc(&tmQ);
-                tma_prefetch_desc(&tmK);
-                tma_prefetch_desc(&tmV);
-                mbar_arrive_expect_tx(BAR(B_QFULL), ntile * C::TILE_BYTES);
-                for (int x = 0; x < ntile; ++x)
-                    for (int pn = 0; pn < C::PANELS; ++pn)
-                        tma_load_3d(sb + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmQ,
-                                    BAR(B_QFULL), pn * 64, h0 + x, row0);
+        if (lane == 0) {
+            tma_prefetch_desc(&tmQ);
+            tma_prefetch_desc(&tmK);
+            tma_prefetch_desc(&tmV);
+        }
+        uint32_t kpos = 0; // position in the K / V ring, running over the items
+        bool live = true;
+        for (int w = 0; live; ++w) {
+            // draw the next item once the queue slot's last reader (four items ago) is done
+            const int slot = w & 3;
+            int idx = -1;
+            if (lane == 0 && mbar_wait(BAR(B_WQFREE + slot), ((w >> 2) & 1) ^ 1, abort_flag)) {
+                idx = atomicAdd(P.cursor, 1);
+                idx = idx < P.n_items ? idx : -1;
+                wq[slot] = idx;
+                mbar_arrive(BAR(B_WQFULL + slot));
             }
+            idx = __shfl_sync(0xffffffffu, idx, 0);
+            if (idx < 0)
+                break;
+            const Item it = decode(idx);
+            const int cnt = it.cnt, n_single = it.n_single, g = it.g;
+            const int2 *klist = it.klist;
+            if (lane == 0) {
+                live = mbar_wait(BAR(B_QEMPTY), (w & 1) ^ 1, abort_flag);
+                if (live) {
+                    mbar_arrive_expect_tx(BAR(B_QFULL), ntile * C::TILE_BYTES);
+                    for (int x = 0; x < ntile; ++x)
+                        for (int pn = 0; pn < C::PANELS; ++pn)
+                            tma_load_3d(sb + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES, &tmQ,
+                                        BAR(B_QFULL), pn * 64, it.h0 + x, it.row0);
+                }
+            }
+            live = __all_sync(0xffffffffu, live);
             // The key tiles of the SINGLE entries go through the same K / V ring first; the softmax
             // warps read their rows from shared memory.
-            bool live = true;
             for (int i = 0; live && i < n_single; ++i) {
-                const int st = i % NS, ph = (i / NS) & 1;
-                const int start = P.sbase[qt * MAX_SINGLE + i];
+                const uint32_t pos = kpos + i;
+                const int st = pos % NS, ph = (pos / NS) & 1;
+                const int start = P.sbase[it.qt * MAX_SINGLE + i];
                 bool ok = true;
                 if (lane == 0) {
                     ok = mbar_wait(BAR(B_KEMPTY + st), ph ^ 1, abort_flag) &&
@@ -204,8 +260,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (cnt > 0)
                 tile_meta(e_cur, m_cur);
             for (int j = 0; live && j < cnt; ++j) {
-                const int jj = n_single + j; // position in the K / V ring
-                const int st = jj % NS, ph = (jj / NS) & 1;
+                const uint32_t pos = kpos + n_single + j;
+                const int st = pos % NS, ph = (pos / NS) & 1;
                 const int start = e_cur.x;
                 const int2 e_nn = j + 2 < cnt ? klist[j + 2] : e_nxt;
                 if (j + 1 < cnt)
@@ -221,7 +277,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                 }
                 ok = ok && mbar_wait(BAR(B_VEMPTY + st), ph ^ 1, abort_flag);
-                if (!__all_sync(0xffffffffu, ok))
+                live = __all_sync(0xffffffffu, ok);
+                if (!live)
                     break;
 #pragma unroll
                 for (int i = 0; i < BN / 32; ++i)
@@ -239,6 +296,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int i = 0; i < BN / 32; ++i)
                     m_cur[i] = m_nxt[i];
             }
+            kpos += (uint32_t)(n_single + cnt);
         }
     } else if (warp == 8 || warp == 10) {
         // ------------------------------------------------------------ MMA issue
@@ -246,7 +304,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // tiles are independent instruction streams (they only share the K / V stages, which are
         // released once both threads have committed), and two threads issue twice as fast as one.
         const int x = (warp - 8) >> 1;
-        if (lane == 0 && cnt > 0 && x < ntile) {
+        if (lane == 0 && x < ntile) {
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, BN, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16_f32(128, D, 0, 1);
             constexpr uint32_t TU = C::TILE_BYTES >> 4, PU = C::PANEL_BYTES >> 4;
@@ -275,48 +333,76 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 tc_commit(BAR(B_PVDONE + x));
                 tc_commit(BAR(B_VEMPTY + st));
             };
-            // Ring positions: the SINGLE entries come first.  Their phases are waited for one by
-            // one: a parity wait is only meaningful on the phase that follows the last one seen.
-            bool ok = mbar_wait(BAR(B_QFULL), 0, abort_flag);
-            for (int i = 0; ok && i < n_single; ++i)
-                ok = mbar_wait(BAR(B_KFULL + i % NS), (i / NS) & 1, abort_flag) &&
-                     mbar_wait(BAR(B_VFULL + i % NS), (i / NS) & 1, abort_flag);
-            ok = ok && mbar_wait(BAR(B_KFULL + n_single % NS), (n_single / NS) & 1, abort_flag);
-            if (ok) {
-                tc_fence_after();
-                issue_s(n_single % NS);
-            }
-            for (int j = 0; ok && j < cnt; ++j) {
-                const int jj = n_single + j;
-                const int st = jj % NS, ph = (jj / NS) & 1;
-                const int nst = (jj + 1) % NS, nph = ((jj + 1) / NS) & 1;
-                const bool more = j + 1 < cnt;
-                if constexpr (C::P_SEPARATE) {
-                    // S(j+1) as soon as the softmax warps hold S(j) in registers
-                    if (more) {
-                        ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag) &&
-                             mbar_wait(BAR(B_SREAD + x), j & 1, abort_flag);
-                        if (!ok)
-                            break;
-                        tc_fence_after();
-                        issue_s(nst);
-                    }
-                }
-                ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag) &&
-                     mbar_wait(BAR(B_PFULL + x), j & 1, abort_flag);
-                if (!ok)
+            uint32_t kpos = 0; // position in the K / V ring, running over the items
+            uint32_t t = 0;    // key tiles of this thread's tile so far (phases of S, P, PV)
+            bool ok = true;
+            for (int w = 0; ok; ++w) {
+                const int idx = take(w);
+                if (idx < 0)
                     break;
-                tc_fence_after();
-                issue_pv(st, j > 0 || n_single > 0);
-                if constexpr (!C::P_SEPARATE) {
-                    // P overwrote S(j): S(j+1) can only follow the P V product that reads it
-                    if (more) {
-                        ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag);
-                        if (!ok)
-                            break;
-                        issue_s(nst);
+                const Item it = decode(idx);
+                const int cnt = it.cnt, n_single = it.n_single;
+                ok = mbar_wait(BAR(B_QFULL), w & 1, abort_flag);
+                // The SINGLE entries come first in the ring.  Their phases are waited for one by
+                // one: a parity wait is only meaningful on the phase that follows the last one
+                // seen.
+                for (int i = 0; ok && i < n_single; ++i) {
+                    const uint32_t pos = kpos + i;
+                    ok = mbar_wait(BAR(B_KFULL + pos % NS), (pos / NS) & 1, abort_flag) &&
+                         mbar_wait(BAR(B_VFULL + pos % NS), (pos / NS) & 1, abort_flag);
+                }
+                if (ok && cnt == 0)
+                    mbar_arrive(BAR(B_QEMPTY)); // no product reads this Q
+                if (ok && cnt > 0) {
+                    const uint32_t p0 = kpos + n_single;
+                    // S of the previous item's last key tile must be in the softmax registers
+                    ok = mbar_wait(BAR(B_KFULL + p0 % NS), (p0 / NS) & 1, abort_flag) &&
+                         (t == 0 || mbar_wait(BAR(B_SREAD + x), (t - 1) & 1, abort_flag));
+                    if (ok) {
+                        tc_fence_after();
+                        issue_s(p0 % NS);
+                        if (cnt == 1)
+                            tc_commit(BAR(B_QEMPTY));
                     }
                 }
+                for (int j = 0; ok && j < cnt; ++j) {
+                    const uint32_t pos = kpos + n_single + j, tt = t + j;
+                    const int st = pos % NS, ph = (pos / NS) & 1;
+                    const int nst = (pos + 1) % NS, nph = ((pos + 1) / NS) & 1;
+                    const bool more = j + 1 < cnt;
+                    if constexpr (C::P_SEPARATE) {
+                        // S(j+1) as soon as the softmax warps hold S(j) in registers
+                        if (more) {
+                            ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag) &&
+                                 mbar_wait(BAR(B_SREAD + x), tt & 1, abort_flag);
+                            if (!ok)
+                                break;
+                            tc_fence_after();
+                            issue_s(nst);
+                            if (j + 2 == cnt)
+                                tc_commit(BAR(B_QEMPTY)); // the item's last product with Q
+                        }
+                    }
+                    ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag) &&
+                         mbar_wait(BAR(B_PFULL + x), tt & 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    issue_pv(st, j > 0 || n_single > 0);
+                    if constexpr (!C::P_SEPARATE) {
+                        // P overwrote S(j): S(j+1) can only follow the P V product that reads it
+                        if (more) {
+                            ok = mbar_wait(BAR(B_KFULL + nst), nph, abort_flag);
+                            if (!ok)
+                                break;
+                            issue_s(nst);
+                            if (j + 2 == cnt)
+                                tc_commit(BAR(B_QEMPTY));
+                        }
+                    }
+                }
+                kpos += (uint32_t)(n_single + cnt);
+                t += (uint32_t)cnt;
             }
         }
     } else if (warp < 4 * ntile) {
@@ -324,24 +410,38 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // ------------------------------------------------------------ softmax of tile x
         const int x = warp >> 2;
         const int r = threadIdx.x & 127;
-        const int h = h0 + x;
-        const int row = row0 + r;
-        const bool row_ok = row < P.q_end;
-        int32_t mq = row_ok ? P.meta[row] : META_NONE_Q;
-        if (mq == META_NONE_K)
-            mq = META_NONE_Q;
         const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t tS = tmem + lane_sel + C::TM_S + x * 128;
         const uint32_t tO = tmem + lane_sel + C::TM_O + x * D;
         const uint32_t tP = tmem + lane_sel + C::TM_P + x * C::P_STRIDE;
-        float m = -CUDART_INF_F, l = 0.f;
+        uint32_t kpos = 0; // position in the K / V ring, running over the items
+        uint32_t t = 0;    // key tiles of this tile so far (phases of S, P, PV)
         bool ok = true;
+        for (int w = 0; ok; ++w) {
+        const int idx = __shfl_sync(0xffffffffu, take(w), 0);
+        __syncwarp();
+        if (lane == 0 && idx >= 0)
+            mbar_arrive(BAR(B_WQFREE + (w & 3))); // this warp has read the queue slot
+        if (idx < 0)
+            break;
+        const Item it = decode(idx);
+        const int qt = it.qt, cnt = it.cnt, n_single = it.n_single;
+        const int2 *klist = it.klist;
+        const int h = it.h0 + x;
+        const int row = it.row0 + r;
+        const bool row_ok = row < P.q_end;
+        int32_t mq = row_ok ? P.meta[row] : META_NONE_Q;
+        if (mq == META_NONE_K)
+            mq = META_NONE_Q;
+        float m = -CUDART_INF_F, l = 0.f;
+        if (n_single == 0 && lane == 0)
+            mbar_arrive(BAR(B_QEMPTY)); // no row of Q is read by this warp
         if constexpr (D == 64) {
             if (n_single > 0) {
                 // One allowed key per row and tile: the score and the weighted value on the CUDA
                 // cores, rows read from the staged K / V tiles, as an online softmax; the result
                 // becomes the starting (m, l, O) of the tile loop.
-                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL), 0, abort_flag));
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL), w & 1, abort_flag));
                 uint32_t qv[32];
                 {
                     const uint8_t *qrow = sp + C::OFF_Q + x * C::TILE_BYTES + r * 128;
@@ -354,12 +454,16 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         qv[4 * c + 3] = v.w;
                     }
                 }
+                __syncwarp();
+                if (lane == 0)
+                    mbar_arrive(BAR(B_QEMPTY)); // this warp's rows of Q are in registers
                 float o[64];
 #pragma unroll
                 for (int i = 0; i < 64; ++i)
                     o[i] = 0.f;
                 for (int i = 0; ok && i < n_single; ++i) {
-                    const int st = i % NS, ph = (i / NS) & 1;
+                    const uint32_t pos = kpos + i;
+                    const int st = pos % NS, ph = (pos / NS) & 1;
                     const int col = P.scs[((size_t)qt * MAX_SINGLE + i) * BM + r];
                     ok = mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
                          mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
@@ -370,12 +474,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const uint4 v = *reinterpret_cast<const uint4 *>(krow + ((c ^ (col & 7)) << 4));
-                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                            const uint32_t kw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
-                                acc = fmaf(__uint_as_float(qv[4 * c + k] << 16), __uint_as_float(w[k] << 16), acc);
+                                acc = fmaf(__uint_as_float(qv[4 * c + k] << 16), __uint_as_float(kw[k] << 16), acc);
                                 acc = fmaf(__uint_as_float(qv[4 * c + k] & 0xffff0000u),
-                                           __uint_as_float(w[k] & 0xffff0000u), acc);
+                                           __uint_as_float(kw[k] & 0xffff0000u), acc);
                             }
                         }
                         const float s2 = acc * P.scale_log2;
@@ -392,12 +496,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const uint4 v = *reinterpret_cast<const uint4 *>(vrow + ((c ^ (col & 7)) << 4));
-                            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+                            const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
-                                o[8 * c + 2 * k] = fmaf(pr, __uint_as_float(w[k] << 16), o[8 * c + 2 * k]);
+                                o[8 * c + 2 * k] = fmaf(pr, __uint_as_float(vw[k] << 16), o[8 * c + 2 * k]);
                                 o[8 * c + 2 * k + 1] =
-                                    fmaf(pr, __uint_as_float(w[k] & 0xffff0000u), o[8 * c + 2 * k + 1]);
+                                    fmaf(pr, __uint_as_float(vw[k] & 0xffff0000u), o[8 * c + 2 * k + 1]);
                             }
                         }
                     }
@@ -424,12 +528,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
         int cls_nxt = cnt > 0 ? klist[0].y >> 16 : 0;
         for (int j = 0; ok && j < cnt; ++j) {
-            const int jj = n_single + j; // position in the K / V ring
-            const int st = jj % NS, ph = (jj / NS) & 1;
+            const uint32_t pos = kpos + n_single + j, tt = t + j;
+            const int st = pos % NS, ph = (pos / NS) & 1;
             const int cls = cls_nxt;
             if (j + 1 < cnt)
                 cls_nxt = klist[j + 1].y >> 16; // used one key tile later
-            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL + x), j & 1, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL + x), tt & 1, abort_flag));
             if (!ok)
                 break;
             tc_fence_after();
@@ -474,7 +578,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 // P V of the previous key tile must be done before O or P are touched
                 if (j > 0) {
                     ok = __all_sync(0xffffffffu,
-                                    mbar_wait(BAR(B_PVDONE + x), (j - 1) & 1, abort_flag));
+                                    mbar_wait(BAR(B_PVDONE + x), (tt - 1) & 1, abort_flag));
                     if (!ok)
                         break;
                     tc_fence_after();
@@ -536,7 +640,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
         } else if (__all_sync(0xffffffffu,
                               ok && (cnt == 0 ||
-                                     mbar_wait(BAR(B_PVDONE + x), (cnt - 1) & 1, abort_flag)))) {
+                                     mbar_wait(BAR(B_PVDONE + x), (t + cnt - 1) & 1, abort_flag)))) {
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
@@ -560,7 +664,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (row_ok)
                 P.LSE[(size_t)h * P.T + row] =
                     l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
+        } else {
+            ok = false; // a wait ran out
         }
+        kpos += (uint32_t)(n_single + cnt);
+        t += (uint32_t)cnt;
+        } // items
     }
 
     // ------------------------------------------------------------ teardown
@@ -601,8 +710,8 @@ int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, in
 }
 
 template <int D>
-static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cudaStream_t s,
-                        cudaEvent_t ev0, cudaEvent_t ev1)
+static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm,
+                        cudaStream_t s, cudaEvent_t ev0, cudaEvent_t ev1)
 {
     CUtensorMap tmQ, tmK, tmV;
     if (make_map(enc, &tmQ, a.Q, D, a.Hq, p.T) || make_map(enc, &tmK, a.K, D, a.Hkv, p.T) ||
@@ -614,6 +723,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
     P.qorder = p.qorder;
     P.meta = p.meta;
     P.status = p.status;
+    P.cursor = p.counters + 3;
     P.n_kt = p.n_kt;
     P.q_begin = p.q_begin;
     P.q_end = p.q_end;
@@ -638,9 +748,10 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
         attr_set = true;
     }
     const int n_hb = P.two ? a.Hq / 2 : a.Hq;
+    P.n_items = p.n_qt * n_hb;
     if (ev0)
         cudaEventRecord(ev0, s);
-    fwd_kernel<D><<<p.n_qt * n_hb, 384, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
+    fwd_kernel<D><<<std::min(P.n_items, n_sm), 384, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
     if (ev1)
         cudaEventRecord(ev1, s);
     return 1;
@@ -649,11 +760,10 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, cuda
 int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
                cudaEvent_t ev0, cudaEvent_t ev1)
 {
-    (void)n_sm;
     if (p.n_qt == 0)
         return 0;
-    return a.D == 64 ? launch_fwd_t<64>(p, a, enc, s, ev0, ev1)
-                     : launch_fwd_t<128>(p, a, enc, s, ev0, ev1);
+    return a.D == 64 ? launch_fwd_t<64>(p, a, enc, n_sm, s, ev0, ev1)
+                     : launch_fwd_t<128>(p, a, enc, n_sm, s, ev0, ev1);
 }
 
 } // namespace peagle
