@@ -1135,10 +1135,14 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
     }
     const size_t n_prep = (size_t)q_len * a.Hq * (D / 8);
     const size_t n_prep_pad = (size_t)q_pad * a.Hq * (D / 8);
-    bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
-        static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.LSE,
-        p.meta, a.nl2, a.nd, a.mqp, a.dq_acc, p.q_begin, q_len, q_pad, a.Hq, p.T);
-    int launches = 1;
+    // Per-row values and the initial dQ staging: with SINGLE tiles, their backward does both.
+    int launches = launch_bwd_single(p, a, s);
+    if (launches == 0) {
+        bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
+            static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.LSE,
+            p.meta, a.nl2, a.nd, a.mqp, a.dq_acc, p.q_begin, q_len, q_pad, a.Hq, p.T);
+        launches = 1;
+    }
     if (p.n_kt > 0) {
         BwdParams P;
         P.ktile = p.ktile;
@@ -1183,7 +1187,6 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
             cudaEventRecord(ev1, s);
         ++launches;
     }
-    launches += launch_bwd_single(p, a, s);
     bwd_finish_dq<<<(unsigned)((n_prep + 255) / 256), 256, 0, s>>>(
         a.dq_acc, static_cast<__nv_bfloat16 *>(a.dQ) + (size_t)p.q_begin * a.Hq * D, n_prep);
     return launches + 1;

@@ -97,7 +97,8 @@ int launch_fwd(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm, cud
                cudaEvent_t ev0, cudaEvent_t ev1);
 int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cudaStream_t s,
                cudaEvent_t ev0, cudaEvent_t ev1);
-// Backward of the SINGLE tiles (adds to the dQ staging and to dK_acc / dV_acc); launches counted.
+// Backward of the SINGLE tiles (head_dim 64 with SINGLE tiles enabled, else returns 0): adds to
+// dK_acc / dV_acc, and prepares the tile kernel's per-row values and the initial dQ staging.
 int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s);
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s);

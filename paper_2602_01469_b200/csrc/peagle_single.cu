@@ -7,8 +7,11 @@
 //   dQ[q,h] += scale * ds * K[k]      dK[k] += scale * ds * Q[q,h]      dV[k] += p * dO[q,h]
 // One kernel, query-major so that no reverse (key -> queries) list is needed: eight lanes per
 // (query row, KV head) hold 8 of the 64 elements each; for every head of the group they form the
-// row's dQ (one fp32 add to the staging row per head) and add into per-key dK / dV sums kept in
-// registers across the heads (one fp32 add per key row at the end).
+// row's dQ and add into per-key dK / dV sums kept in registers across the heads (one fp32 add per
+// key row at the end).  The kernel runs before the tile kernel and doubles as its preparation
+// pass: it reads O and LSE as well, writes -LSE * log2(e), -Delta and the packed metadata of
+// every row, and its dQ becomes the initial value of the fp32 staging row (plain stores; zero for
+// a row without SINGLE keys), so the staging is never cleared or re-read for these pairs.
 #include <math_constants.h>
 
 #include "peagle_internal.h"
@@ -21,10 +24,13 @@ struct SingleParams {
     const int *scount;
     const uint8_t *scs;  // [n_qt][MAX_SINGLE][BM] key column of entry i for row r, or NO_COL
     const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
-    const __nv_bfloat16 *Q, *K, *V, *dO;
-    const float *nl2, *nd; // [Hq][q_pad]
+    const __nv_bfloat16 *Q, *K, *V, *O, *dO;
+    const float *LSE;      // [Hq][T]
+    const int32_t *meta;   // [T] packed metadata
+    float *nl2, *nd;       // [Hq][q_pad], written here
+    int32_t *mqp;          // [q_pad], written here
     float *dq_acc, *dK_acc, *dV_acc;
-    int q_begin, q_end, q_pad, n_qt, Hq, Hkv;
+    int q_begin, q_end, q_pad, n_qt, Hq, Hkv, T;
     float scale, scale_log2;
 };
 
@@ -66,22 +72,19 @@ __device__ __forceinline__ void red_chunk(float *dst, const float (&x)[8], float
                  : "memory");
 }
 
-// Unit (row r of the partition, KV head g) = 8 lanes; a block of 128 threads holds 16 units.
-// Keys are taken KEYS at a time so that their dK / dV sums fit in registers.
-__global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
+// Unit (row r of the padded partition, KV head g) = 8 lanes; a block of 128 threads holds 16
+// units.  The kernel runs before the tile kernel and also prepares what that kernel needs per
+// (row, head): -LSE * log2(e), -Delta = -<dO, O>, the row's packed metadata, and the initial value
+// of the fp32 dQ staging row, which is this kernel's own contribution (zero for a row without
+// SINGLE keys), written with plain stores.  Keys are taken KEYS at a time so that their dK / dV
+// sums fit in registers; a row with more than KEYS keys adds its later groups with reductions.
+// One pass over KEYS of the row's SINGLE keys, all heads of the group.  The first pass also
+// prepares the row (FIRST) and stores its dQ; later passes add theirs.
+template <bool FIRST, int KEYS>
+__device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int ns, int sub, unsigned um,
+                                            int r, int g, int row, int qt, int rr, int G, size_t qoff)
 {
-    constexpr int KEYS = 4;
-    const int sub = threadIdx.x & 7;
-    const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
-    const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
-    const int r = (int)(unit / P.Hkv), g = (int)(unit % P.Hkv);
-    const int row = P.q_begin + r;
-    if (row >= P.q_end)
-        return; // the 8 lanes of a unit leave together
-    const int qt = r / BM, rr = r % BM;
-    const int ns = min(P.scount[qt], MAX_SINGLE);
-    const int G = P.Hq / P.Hkv;
-    for (int i0 = 0; i0 < ns; i0 += KEYS) {
+        constexpr bool first = FIRST;
         int tok[KEYS];
         bool any = false;
 #pragma unroll
@@ -94,8 +97,8 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
             }
             any |= tok[i] >= 0;
         }
-        if (!any)
-            continue;
+        if (!any && !first)
+            return;
         float dk[KEYS][8], dv[KEYS][8];
         uint4 kp[KEYS], vp[KEYS]; // the keys' elements of this lane, packed bf16
 #pragma unroll
@@ -110,20 +113,51 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
             }
         }
         // the rows of the next head are requested before this head's arithmetic
-        const size_t qoff = ((size_t)row * P.Hq + (size_t)g * G) * 64;
         uint4 qn = reinterpret_cast<const uint4 *>(P.Q + qoff)[sub];
         uint4 dn = reinterpret_cast<const uint4 *>(P.dO + qoff)[sub];
-        float nl2n = P.nl2[(size_t)(g * G) * P.q_pad + r], ndn = P.nd[(size_t)(g * G) * P.q_pad + r];
+        uint4 on = make_uint4(0, 0, 0, 0);
+        float ln = 0.f; // first pass: LSE; later passes: the stored -LSE * log2(e)
+        float ndn = 0.f;
+        if (first) {
+            on = reinterpret_cast<const uint4 *>(P.O + qoff)[sub];
+            ln = P.LSE[(size_t)(g * G) * P.T + row];
+        } else { // written by lane 0 of this unit in the first pass: read past L1
+            ln = __ldcg(P.nl2 + (size_t)(g * G) * P.q_pad + r);
+            ndn = __ldcg(P.nd + (size_t)(g * G) * P.q_pad + r);
+        }
         for (int hh = 0; hh < G; ++hh) {
             const int h = g * G + hh;
-            const float nl2 = nl2n, nd = ndn;
+            const float lcur = ln;
+            float nd = ndn;
             const Chunk q = unpack_chunk(qn);
             const Chunk dO = unpack_chunk(dn);
+            const Chunk o = unpack_chunk(on);
             if (hh + 1 < G) {
                 qn = reinterpret_cast<const uint4 *>(P.Q + qoff + (size_t)(hh + 1) * 64)[sub];
                 dn = reinterpret_cast<const uint4 *>(P.dO + qoff + (size_t)(hh + 1) * 64)[sub];
-                nl2n = P.nl2[(size_t)(h + 1) * P.q_pad + r];
-                ndn = P.nd[(size_t)(h + 1) * P.q_pad + r];
+                if (first) {
+                    on = reinterpret_cast<const uint4 *>(P.O + qoff + (size_t)(hh + 1) * 64)[sub];
+                    ln = P.LSE[(size_t)(h + 1) * P.T + row];
+                } else {
+                    ln = __ldcg(P.nl2 + (size_t)(h + 1) * P.q_pad + r);
+                    ndn = __ldcg(P.nd + (size_t)(h + 1) * P.q_pad + r);
+                }
+            }
+            float nl2 = lcur;
+            if (first) {
+                float delta = 0.f;
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    delta = fmaf(dO.v[e], o.v[e], delta);
+#pragma unroll
+                for (int s = 1; s < 8; s <<= 1)
+                    delta += __shfl_xor_sync(um, delta, s);
+                nd = -delta;
+                nl2 = lcur == -CUDART_INF_F ? -CUDART_INF_F : -lcur * 1.4426950408889634f;
+                if (sub == 0) {
+                    P.nl2[(size_t)h * P.q_pad + r] = nl2;
+                    P.nd[(size_t)h * P.q_pad + r] = nd;
+                }
             }
             float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -139,9 +173,9 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
                     dp = fmaf(dO.v[e], v.v[e], dp);
                 }
 #pragma unroll
-                for (int o = 1; o < 8; o <<= 1) {
-                    s += __shfl_xor_sync(um, s, o);
-                    dp += __shfl_xor_sync(um, dp, o);
+                for (int o2 = 1; o2 < 8; o2 <<= 1) {
+                    s += __shfl_xor_sync(um, s, o2);
+                    dp += __shfl_xor_sync(um, dp, o2);
                 }
                 const float p = fast_exp2(fmaf(s, P.scale_log2, nl2)); // nl2 = -inf: p = 0
                 const float ds = p * (dp + nd);
@@ -152,7 +186,15 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
                     dv[i][e] = fmaf(p, dO.v[e], dv[i][e]);
                 }
             }
-            red_chunk(P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8, dq, P.scale);
+            float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8;
+            if (first) {
+                reinterpret_cast<float4 *>(dst)[0] = make_float4(dq[0] * P.scale, dq[1] * P.scale,
+                                                                 dq[2] * P.scale, dq[3] * P.scale);
+                reinterpret_cast<float4 *>(dst)[1] = make_float4(dq[4] * P.scale, dq[5] * P.scale,
+                                                                 dq[6] * P.scale, dq[7] * P.scale);
+            } else {
+                red_chunk(dst, dq, P.scale);
+            }
         }
 #pragma unroll
         for (int i = 0; i < KEYS; ++i)
@@ -161,6 +203,41 @@ __global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
                 red_chunk(P.dK_acc + kr, dk[i], P.scale);
                 red_chunk(P.dV_acc + kr, dv[i], 1.f);
             }
+}
+
+__global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
+{
+    constexpr int KEYS = 4;
+    const int sub = threadIdx.x & 7;
+    const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
+    const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
+    const int r = (int)(unit / P.Hkv), g = (int)(unit % P.Hkv);
+    if (r >= P.q_pad)
+        return; // the 8 lanes of a unit leave together
+    const int row = P.q_begin + r;
+    const int G = P.Hq / P.Hkv;
+    if (row >= P.q_end) { // padded row: seen by nobody
+        if (sub == 0) {
+            for (int hh = 0; hh < G; ++hh) {
+                P.nl2[(size_t)(g * G + hh) * P.q_pad + r] = -CUDART_INF_F;
+                P.nd[(size_t)(g * G + hh) * P.q_pad + r] = 0.f;
+            }
+            if (g == 0)
+                P.mqp[r] = META_NONE_Q;
+        }
+        return;
+    }
+    if (g == 0 && sub == 0) {
+        const int32_t mq = P.meta[row];
+        P.mqp[r] = mq == META_NONE_K ? META_NONE_Q : mq;
+    }
+    const int qt = r / BM, rr = r % BM;
+    const int ns = min(P.scount[qt], MAX_SINGLE);
+    const size_t qoff = ((size_t)row * P.Hq + (size_t)g * G) * 64;
+    single_pass<true, KEYS>(P, 0, ns, sub, um, r, g, row, qt, rr, G, qoff);
+    for (int i0 = KEYS; i0 < ns; i0 += KEYS) {
+        __syncwarp(um); // lane 0's row values are visible to the unit's later passes
+        single_pass<false, KEYS>(P, i0, ns, sub, um, r, g, row, qt, rr, G, qoff);
     }
 }
 
@@ -175,9 +252,13 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);
+    P.O = static_cast<const __nv_bfloat16 *>(a.O);
     P.dO = static_cast<const __nv_bfloat16 *>(a.dO);
+    P.LSE = a.LSE;
+    P.meta = p.meta;
     P.nl2 = a.nl2;
     P.nd = a.nd;
+    P.mqp = a.mqp;
     P.dq_acc = a.dq_acc;
     P.dK_acc = a.dK_acc;
     P.dV_acc = a.dV_acc;
@@ -187,9 +268,10 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.n_qt = p.n_qt;
     P.Hq = a.Hq;
     P.Hkv = a.Hkv;
+    P.T = p.T;
     P.scale = a.scale;
     P.scale_log2 = a.scale * 1.4426950408889634f;
-    const size_t units = (size_t)(p.q_end - p.q_begin) * a.Hkv; // of 8 lanes each
+    const size_t units = (size_t)P.q_pad * a.Hkv; // of 8 lanes each
     single_bwd<<<(unsigned)((units + 15) / 16), 128, 0, s>>>(P);
     return 1;
 }
