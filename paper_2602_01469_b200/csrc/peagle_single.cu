@@ -162,8 +162,6 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
             float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < KEYS; ++i) {
-                if (tok[i] < 0)
-                    continue; // same for the 8 lanes of the unit
                 const Chunk k = unpack_chunk(kp[i]);
                 const Chunk v = unpack_chunk(vp[i]);
                 float s = 0.f, dp = 0.f;
@@ -177,7 +175,9 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
                     s += __shfl_xor_sync(um, s, o2);
                     dp += __shfl_xor_sync(um, dp, o2);
                 }
-                const float p = fast_exp2(fmaf(s, P.scale_log2, nl2)); // nl2 = -inf: p = 0
+                // an absent key takes part with weight zero, so that the keys' chains of dependent
+                // instructions interleave instead of branching around each other
+                const float p = fast_exp2(fmaf(s, P.scale_log2, tok[i] >= 0 ? nl2 : -CUDART_INF_F)); // nl2 = -inf: p = 0
                 const float ds = p * (dp + nd);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -205,9 +205,12 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
             }
 }
 
-__global__ void __launch_bounds__(128) single_bwd(const SingleParams P)
+// Two keys per pass and four resident blocks per SM (128 registers): the kernel is bound by the
+// latency of its dependent chains (dot product, three shuffles, exp2), so more warps pay more
+// than fewer passes; four keys per pass at two blocks per SM was 20 % slower.
+__global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
 {
-    constexpr int KEYS = 4;
+    constexpr int KEYS = 2;
     const int sub = threadIdx.x & 7;
     const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
     const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
