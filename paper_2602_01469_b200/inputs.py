@@ -156,6 +156,17 @@ def make_tensors(T: int, Hq: int, Hkv: int, D: int, seed: int, q_std: float | No
     return tuple(out)  # Q, K, V, dO
 
 
+def make_fused_rows(T: int, Hq: int, Hkv: int, D: int, seed: int):
+    """bf16 fused projection rows [T, (Hq + 2 Hkv) * D] ~ N(0,1) (the rotary prologue's input) and
+    bf16 upstream gradients dQ [T, Hq, D], dK, dV [T, Hkv, D] ~ N(0,1) for its backward."""
+    out = []
+    for i, shape in enumerate(((T, (Hq + 2 * Hkv) * D), (T, Hq, D), (T, Hkv, D), (T, Hkv, D))):
+        g = torch.Generator(device="cpu")
+        g.manual_seed(seed * 10 + 5 + i)
+        out.append(torch.randn(*shape, generator=g, dtype=torch.float32).to(torch.bfloat16))
+    return tuple(out)  # qkv, dQ, dK, dV
+
+
 def build_case(w: Workload, assign_fn):
     """Lays out a workload: per sequence the full grid of anchors x depths, segments from
     ``assign_fn(anchor, depth, K, boundaries) -> segment per token`` (Algorithm 1, supplied by the
