@@ -312,6 +312,57 @@ def run_cuda(args, w):
         dist.destroy_process_group()
 
 
+def run_rope(args, w):
+    """The rotary prologue and its backward on the workload's token grid: an HBM-bound side line
+    (one read and one write of every element per direction), timed with CUDA events."""
+    import torch
+
+    from paper_2602_01469_b200 import binding
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    cu, anchor, depth, _ = inputs.build_case(w, binding.peagle_assign_segments)
+    T, Hq, Hkv, D = int(cu[-1]), w.n_q_heads, w.n_kv_heads, w.head_dim
+    qkv, gQ, gK, gV = (t.to(dev) for t in inputs.make_fused_rows(T, Hq, Hkv, D, w.seed))
+    d_anchor, d_depth = torch.from_numpy(anchor).to(dev), torch.from_numpy(depth).to(dev)
+    Q, K, V, gx = torch.empty_like(gQ), torch.empty_like(gK), torch.empty_like(gV), torch.empty_like(qkv)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.peagle_rope_qkv_fwd(ctx, qkv, d_anchor, d_depth, Hq, Hkv, D, 500000.0, Q, K, V, stream)
+        binding.peagle_rope_qkv_bwd(ctx, gQ, gK, gV, d_anchor, d_depth, Hq, Hkv, D, 500000.0, gx, stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(0) as clocks:
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    # per direction: every element of the fused row read once and written once, 8 bytes of metadata
+    bytes_step = 2 * (2 * qkv.numel() * 2 + 8 * T)
+    peaks, src = load_peaks()
+    peak = float(peaks["hbm_gbs"])
+    gbs = bytes_step / (ms * 1e-3) / 1e9
+    print(json.dumps({
+        "metric": "rotary prologue fwd+bwd GB/s", "value": gbs, "unit": "GB/s", "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "total_tokens": T, "n_q_heads": Hq, "n_kv_heads": Hkv,
+                   "head_dim": D, "l2": "tensors (%.2f GB) larger than L2, no flush" % (bytes_step / 2e9)},
+        "clocks": clocks.summary(), "gpu_launches": 2 * args.steps,
+        "roofline": {"kernel": "rope_kernel", "bound": "hbm", "achieved": gbs, "peak": peak,
+                     "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                     "peak_source": "%s hbm_gbs" % src},
+    }))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -319,6 +370,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=inputs.HEADLINE, choices=sorted(inputs.WORKLOADS))
+    ap.add_argument("--op", default="attention", choices=["attention", "rope"],
+                    help="attention: the hot path (default); rope: the rotary prologue side line")
     ap.add_argument("--cpu-seconds", type=float, default=15.0,
                     help="CPU time for the oracle baseline (0 = skip)")
     args = ap.parse_args()
@@ -326,6 +379,8 @@ def main():
     w = inputs.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)
+    elif args.op == "rope":
+        run_rope(args, w)
     else:
         run_cuda(args, w)
 

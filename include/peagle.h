@@ -203,6 +203,32 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
                                  void *dQ, void *dK, void *dV);
 
 /*
+ * Rotary prologue of the drafter layer (Section 2: a LLaMA-3-style layer with rotary position
+ * embeddings; Section 3: the token with anchor a and depth d stands at sequence position a + d).
+ * qkv is dev [total_tokens][(n_q_heads + 2 n_kv_heads) * head_dim] bf16, one fused projection row
+ * per token: query heads, then key heads, then value heads.  Writes the tensors the attention
+ * entry points read: Q [T][Hq][D] and K [T][Hkv][D] with every head turned by the rotation of its
+ * token's position (element i pairs with element i + D/2; angle = position * rope_base^(-2i/D)),
+ * V [T][Hkv][D] copied.  anchor / depth are dev [total_tokens].  All pointers 16-byte aligned;
+ * head_dim 64 or 128; rope_base > 1 (LLaMA 3 uses 500000).  Asynchronous on `stream`; nothing is
+ * allocated.  Buffers are the caller's; in and out must not overlap.  total_tokens == 0 returns
+ * PEAGLE_OK without looking at the pointers; a bad shape or base is PEAGLE_ERR_BAD_SHAPE.
+ */
+int peagle_rope_qkv_fwd(peagle_ctx *ctx, const void *qkv, const int32_t *anchor, const int32_t *depth,
+                        int32_t total_tokens, int32_t n_q_heads, int32_t n_kv_heads,
+                        int32_t head_dim, float rope_base, void *Q, void *K, void *V, void *stream);
+
+/*
+ * Backward of the prologue: the gradients of Q and K are turned back by the inverse rotation and
+ * packed with the gradient of V into d_qkv, the gradient of the fused row (same layout as qkv).
+ * Same argument rules as the forward.
+ */
+int peagle_rope_qkv_bwd(peagle_ctx *ctx, const void *dQ, const void *dK, const void *dV,
+                        const int32_t *anchor, const int32_t *depth, int32_t total_tokens,
+                        int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float rope_base,
+                        void *d_qkv, void *stream);
+
+/*
  * Algorithm 1, host only: segment of every token.  `boundaries` is host [S+1], context-token
  * positions with boundaries[0]=0 and boundaries[S]=n (Algorithm 1's B).  Depth 0 and 1 tokens
  * go by their position anchor+depth (a position at or beyond n stays in the last segment);

@@ -26,6 +26,7 @@ EXPORTS = [
     "peagle_attn_bwd", "peagle_attn_partitioned", "peagle_attn_partitioned_host",
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
     "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
+    "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd",
 ]
 
 
@@ -224,6 +225,21 @@ def peagle_attn_partitioned_host(ctx, prob: Problem, parts, Q, K, V, dO, O, LSE,
     _check(lib().peagle_attn_partitioned_host(ctx.h, prob.ref(), arr, len(parts), _ptr(Q), _ptr(K),
                                               _ptr(V), _ptr(dO), _ptr(O), _ptr(LSE), _ptr(dQ),
                                               _ptr(dK), _ptr(dV)), ctx.h)
+
+
+def peagle_rope_qkv_fwd(ctx, qkv, anchor, depth, Hq, Hkv, D, rope_base, Q, K, V, stream=None):
+    """Rotary prologue: fused rows [T, (Hq + 2 Hkv) * D] -> Q, K (rotated), V (copied); device tensors."""
+    _check(lib().peagle_rope_qkv_fwd(ctx.h, _ptr(qkv), _ptr(anchor), _ptr(depth),
+                                     int(qkv.shape[0]), int(Hq), int(Hkv), int(D),
+                                     ctypes.c_float(rope_base), _ptr(Q), _ptr(K), _ptr(V),
+                                     _stream(stream)), ctx.h)
+
+
+def peagle_rope_qkv_bwd(ctx, dQ, dK, dV, anchor, depth, Hq, Hkv, D, rope_base, d_qkv, stream=None):
+    """Backward of the rotary prologue: dQ, dK, dV -> gradient of the fused rows; device tensors."""
+    _check(lib().peagle_rope_qkv_bwd(ctx.h, _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(anchor), _ptr(depth),
+                                     int(dQ.shape[0]), int(Hq), int(Hkv), int(D),
+                                     ctypes.c_float(rope_base), _ptr(d_qkv), _stream(stream)), ctx.h)
 
 
 def peagle_assign_segments(anchor, depth, K, boundaries):

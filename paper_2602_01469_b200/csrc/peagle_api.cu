@@ -515,6 +515,60 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
     return run_fwd(ctx, prob, c, Q, K, V, O, LSE, s);
 }
 
+static int rope_args_ok(int32_t T, int32_t Hq, int32_t Hkv, int32_t D, float base)
+{
+    if (T < 0 || Hq <= 0 || Hkv <= 0 || (D != 64 && D != 128) || !(base > 1.f))
+        return PEAGLE_ERR_BAD_SHAPE;
+    return PEAGLE_OK;
+}
+
+int peagle_rope_qkv_fwd(peagle_ctx *ctx, const void *qkv, const int32_t *anchor, const int32_t *depth,
+                        int32_t total_tokens, int32_t n_q_heads, int32_t n_kv_heads,
+                        int32_t head_dim, float rope_base, void *Q, void *K, void *V, void *stream)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    const int rc = rope_args_ok(total_tokens, n_q_heads, n_kv_heads, head_dim, rope_base);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (total_tokens == 0)
+        return PEAGLE_OK; // nothing to do, pointers not looked at
+    if (!qkv || !anchor || !depth || !Q || !K || !V)
+        return PEAGLE_ERR_NULL;
+    if (!aligned16(qkv) || !aligned16(Q) || !aligned16(K) || !aligned16(V))
+        return PEAGLE_ERR_ALIGN;
+    CK(cudaSetDevice(ctx->device));
+    ctx->launches += launch_rope(false, qkv, nullptr, nullptr, nullptr, nullptr, Q, K, V, anchor, depth,
+                                 total_tokens, n_q_heads, n_kv_heads, head_dim, rope_base,
+                                 ctx->n_sm, static_cast<cudaStream_t>(stream));
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int peagle_rope_qkv_bwd(peagle_ctx *ctx, const void *dQ, const void *dK, const void *dV,
+                        const int32_t *anchor, const int32_t *depth, int32_t total_tokens,
+                        int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, float rope_base,
+                        void *d_qkv, void *stream)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    const int rc = rope_args_ok(total_tokens, n_q_heads, n_kv_heads, head_dim, rope_base);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (total_tokens == 0)
+        return PEAGLE_OK;
+    if (!dQ || !dK || !dV || !anchor || !depth || !d_qkv)
+        return PEAGLE_ERR_NULL;
+    if (!aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(d_qkv))
+        return PEAGLE_ERR_ALIGN;
+    CK(cudaSetDevice(ctx->device));
+    ctx->launches += launch_rope(true, nullptr, d_qkv, dQ, dK, dV, nullptr, nullptr, nullptr, anchor,
+                                 depth, total_tokens, n_q_heads, n_kv_heads, head_dim, rope_base,
+                                 ctx->n_sm, static_cast<cudaStream_t>(stream));
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
 int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,
                            const peagle_partition_t *part, const void *Q, const void *K,
                            const void *V, void *O, float *LSE, int32_t *dev_status, void *stream)

@@ -103,6 +103,13 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s);
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s);
 
+// Rotary prologue (backward = false: fused row -> Q, K, V) and its backward (dQ, dK, dV -> gradient
+// of the fused row).  Returns the number of kernels launched.
+int launch_rope(bool backward, const void *fused_in, void *fused_out, const void *q_in,
+                const void *k_in, const void *v_in, void *q_out, void *k_out, void *v_out,
+                const int32_t *anchor, const int32_t *depth, int T, int Hq, int Hkv, int D,
+                float base, int n_sm, cudaStream_t s);
+
 // Packed-metadata form of the attention predicate: m = anchor << 8 | depth.
 // (depth_k == 0 and anchor_k <= anchor_q) or (anchor_k == anchor_q and depth_k <= depth_q)
 __host__ __device__ inline bool allowed_packed(int32_t mq, int32_t mk)
