@@ -26,7 +26,6 @@ using namespace sm100;
 namespace {
 
 constexpr int ROPE_THREADS = 256;
-constexpr int ROPE_TOKENS = 2; // tokens per block iteration
 
 struct RopeParams {
     const __nv_bfloat16 *fused_in;          // forward: [T][(Hq + 2 Hkv) * D]
@@ -59,6 +58,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kernel(const RopeParams P)
 {
     constexpr int HALF = D / 2;
     constexpr int CH = D / 16; // 16-byte pieces per half head = tasks per head
+    constexpr int ROPE_TOKENS = ROPE_THREADS / HALF; // tokens per iteration: a table entry per thread
     __shared__ float s_cos[ROPE_TOKENS][HALF], s_sin[ROPE_TOKENS][HALF];
     const int heads = P.Hq + 2 * P.Hkv;
     const int tasks = heads * CH; // per token
@@ -134,7 +134,7 @@ __global__ void __launch_bounds__(ROPE_THREADS) rope_kernel(const RopeParams P)
 template <int D, bool BACKWARD>
 int launch_rope_t(const RopeParams &P, int n_sm, cudaStream_t s)
 {
-    static_assert(ROPE_THREADS >= ROPE_TOKENS * (D / 2), "one thread per (token, pair) of the tables");
+    constexpr int ROPE_TOKENS = ROPE_THREADS / (D / 2);
     const int blocks = std::min((P.T + ROPE_TOKENS - 1) / ROPE_TOKENS, n_sm * 8);
     rope_kernel<D, BACKWARD><<<blocks, ROPE_THREADS, 0, s>>>(P);
     return 1;
