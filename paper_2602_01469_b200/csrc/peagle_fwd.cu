@@ -442,16 +442,18 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 // cores, rows read from the staged K / V tiles, as an online softmax; the result
                 // becomes the starting (m, l, O) of the tile loop.
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL), w & 1, abort_flag));
-                uint32_t qv[32];
+                float qf[64]; // the row of Q, unpacked once
                 {
                     const uint8_t *qrow = sp + C::OFF_Q + x * C::TILE_BYTES + r * 128;
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         const uint4 v = *reinterpret_cast<const uint4 *>(qrow + ((c ^ (r & 7)) << 4));
-                        qv[4 * c] = v.x;
-                        qv[4 * c + 1] = v.y;
-                        qv[4 * c + 2] = v.z;
-                        qv[4 * c + 3] = v.w;
+                        const uint32_t qw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            qf[8 * c + 2 * k] = __uint_as_float(qw[k] << 16);
+                            qf[8 * c + 2 * k + 1] = __uint_as_float(qw[k] & 0xffff0000u);
+                        }
                     }
                 }
                 __syncwarp();
@@ -461,29 +463,35 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int i = 0; i < 64; ++i)
                     o[i] = 0.f;
+                int col_nxt = P.scs[((size_t)qt * MAX_SINGLE) * BM + r];
                 for (int i = 0; ok && i < n_single; ++i) {
                     const uint32_t pos = kpos + i;
                     const int st = pos % NS, ph = (pos / NS) & 1;
-                    const int col = P.scs[((size_t)qt * MAX_SINGLE + i) * BM + r];
+                    const int col = col_nxt;
+                    if (i + 1 < n_single) // requested one entry ahead of its use
+                        col_nxt = P.scs[((size_t)qt * MAX_SINGLE + i + 1) * BM + r];
                     ok = mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
                          mbar_wait(BAR(B_VFULL + st), ph, abort_flag);
                     if (ok && col != NO_COL && row_ok) {
                         const uint8_t *krow = sp + C::OFF_K + st * C::TILE_BYTES + col * 128;
                         const uint8_t *vrow = sp + C::OFF_V + st * C::TILE_BYTES + col * 128;
-                        float acc = 0.f;
+                        float acc4[4] = {0.f, 0.f, 0.f, 0.f}; // four chains of dependent adds
 #pragma unroll
                         for (int c = 0; c < 8; ++c) {
                             const uint4 v = *reinterpret_cast<const uint4 *>(krow + ((c ^ (col & 7)) << 4));
                             const uint32_t kw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                             for (int k = 0; k < 4; ++k) {
-                                acc = fmaf(__uint_as_float(qv[4 * c + k] << 16), __uint_as_float(kw[k] << 16), acc);
-                                acc = fmaf(__uint_as_float(qv[4 * c + k] & 0xffff0000u),
-                                           __uint_as_float(kw[k] & 0xffff0000u), acc);
+                                acc4[k] = fmaf(qf[8 * c + 2 * k], __uint_as_float(kw[k] << 16), acc4[k]);
+                                acc4[k] = fmaf(qf[8 * c + 2 * k + 1], __uint_as_float(kw[k] & 0xffff0000u),
+                                               acc4[k]);
                             }
                         }
-                        const float s2 = acc * P.scale_log2;
-                        if (s2 > m) { // bring the running sums to the new maximum
+                        const float s2 = ((acc4[0] + acc4[1]) + (acc4[2] + acc4[3])) * P.scale_log2;
+                        // As in the tile loop, the running sums move to a new maximum only when it
+                        // grew by more than 2^8 (always for the first key, where m is -inf and
+                        // the sums are still zero).
+                        if (s2 > m + 8.f) {
                             const float alpha = fast_exp2(m - s2); // 0 for the first key
                             l *= alpha;
 #pragma unroll
