@@ -14,6 +14,8 @@
 // a row without SINGLE keys), so the staging is never cleared or re-read for these pairs.
 #include <math_constants.h>
 
+#include <algorithm>
+
 #include "peagle_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -30,7 +32,8 @@ struct SingleParams {
     float *nl2, *nd;       // [Hq][q_pad], written here
     int32_t *mqp;          // [q_pad], written here
     float *dq_acc, *dK_acc, *dV_acc;
-    int q_begin, q_end, q_pad, n_qt, Hq, Hkv, T;
+    int *status;
+    int q_begin, q_end, q_pad, n_qt, Hq, Hkv, T, rows_per_block;
     float scale, scale_log2;
 };
 
@@ -78,148 +81,167 @@ __device__ __forceinline__ void red_chunk(float *dst, const float (&x)[8], float
 // of the fp32 dQ staging row, which is this kernel's own contribution (zero for a row without
 // SINGLE keys), written with plain stores.  Keys are taken KEYS at a time so that their dK / dV
 // sums fit in registers; a row with more than KEYS keys adds its later groups with reductions.
-// One pass over KEYS of the row's SINGLE keys, all heads of the group.  The first pass also
-// prepares the row (FIRST) and stores its dQ; later passes add theirs.
+// Block = RB rows of the padded partition x all KV heads; unit (row, KV head g) = 8 lanes.  The
+// rows of Q, dO and O (all heads of a row are contiguous) come in by bulk copies, so that the
+// memory system sees the block's whole input at once instead of one 16-byte load per lane and
+// head; the arithmetic then reads shared memory.  The kernel runs before the tile kernel and
+// also prepares what that kernel needs per (row, head): -LSE * log2(e), -Delta = -<dO, O>, the
+// row's packed metadata, and the initial value of the fp32 dQ staging row, which is this kernel's
+// own contribution (zero for a row without SINGLE keys), written with plain stores.  Keys are
+// taken KEYS at a time so that their dK / dV sums fit in registers; a row with more than KEYS
+// keys adds its later groups with reductions.
 template <bool FIRST, int KEYS>
 __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int ns, int sub, unsigned um,
-                                            int r, int g, int row, int qt, int rr, int G, size_t qoff)
+                                            int r, int g, int qt, int rr, int G,
+                                            const __nv_bfloat16 *sq, const __nv_bfloat16 *sdo,
+                                            const __nv_bfloat16 *so, float *snl2, float *snd)
 {
-        constexpr bool first = FIRST;
-        int tok[KEYS];
-        bool any = false;
+    int tok[KEYS];
+    bool any = false;
 #pragma unroll
-        for (int i = 0; i < KEYS; ++i) {
-            tok[i] = -1;
-            if (i0 + i < ns) {
-                const int col = P.scs[((size_t)qt * MAX_SINGLE + i0 + i) * BM + rr];
-                if (col != NO_COL)
-                    tok[i] = P.sbase[qt * MAX_SINGLE + i0 + i] + col;
-            }
-            any |= tok[i] >= 0;
+    for (int i = 0; i < KEYS; ++i) {
+        tok[i] = -1;
+        if (i0 + i < ns) {
+            const int col = P.scs[((size_t)qt * MAX_SINGLE + i0 + i) * BM + rr];
+            if (col != NO_COL)
+                tok[i] = P.sbase[qt * MAX_SINGLE + i0 + i] + col;
         }
-        if (!any && !first)
-            return;
-        float dk[KEYS][8], dv[KEYS][8];
-        uint4 kp[KEYS], vp[KEYS]; // the keys' elements of this lane, packed bf16
+        any |= tok[i] >= 0;
+    }
+    if (!any && !FIRST)
+        return;
+    float dk[KEYS][8], dv[KEYS][8];
+    uint4 kp[KEYS], vp[KEYS]; // the keys' elements of this lane, packed bf16
+#pragma unroll
+    for (int i = 0; i < KEYS; ++i) {
+        const size_t kr = ((size_t)(tok[i] >= 0 ? tok[i] : 0) * P.Hkv + g) * 64;
+        kp[i] = reinterpret_cast<const uint4 *>(P.K + kr)[sub];
+        vp[i] = reinterpret_cast<const uint4 *>(P.V + kr)[sub];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            dk[i][e] = 0.f;
+            dv[i][e] = 0.f;
+        }
+    }
+    for (int hh = 0; hh < G; ++hh) {
+        const int h = g * G + hh;
+        const Chunk q = load_chunk(sq + (size_t)h * 64, sub);
+        const Chunk dO = load_chunk(sdo + (size_t)h * 64, sub);
+        float nl2, nd;
+        if (FIRST) {
+            const Chunk o = load_chunk(so + (size_t)h * 64, sub);
+            float delta = 0.f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e)
+                delta = fmaf(dO.v[e], o.v[e], delta);
+#pragma unroll
+            for (int s = 1; s < 8; s <<= 1)
+                delta += __shfl_xor_sync(um, delta, s);
+            nd = -delta;
+            const float lse = snl2[h]; // holds LSE until here
+            nl2 = lse == -CUDART_INF_F ? -CUDART_INF_F : -lse * 1.4426950408889634f;
+            __syncwarp(um); // every lane has read the LSE before it is replaced
+            if (sub == 0) {
+                snl2[h] = nl2;
+                snd[h] = nd;
+                P.nl2[(size_t)h * P.q_pad + r] = nl2;
+                P.nd[(size_t)h * P.q_pad + r] = nd;
+            }
+        } else {
+            nl2 = snl2[h];
+            nd = snd[h];
+        }
+        float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
         for (int i = 0; i < KEYS; ++i) {
-            const size_t kr = ((size_t)(tok[i] >= 0 ? tok[i] : 0) * P.Hkv + g) * 64;
-            kp[i] = reinterpret_cast<const uint4 *>(P.K + kr)[sub];
-            vp[i] = reinterpret_cast<const uint4 *>(P.V + kr)[sub];
+            const Chunk k = unpack_chunk(kp[i]);
+            const Chunk v = unpack_chunk(vp[i]);
+            float s = 0.f, dp = 0.f;
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
-                dk[i][e] = 0.f;
-                dv[i][e] = 0.f;
+                s = fmaf(q.v[e], k.v[e], s);
+                dp = fmaf(dO.v[e], v.v[e], dp);
+            }
+#pragma unroll
+            for (int o2 = 1; o2 < 8; o2 <<= 1) {
+                s += __shfl_xor_sync(um, s, o2);
+                dp += __shfl_xor_sync(um, dp, o2);
+            }
+            // an absent key takes part with weight zero, so that the keys' chains of dependent
+            // instructions interleave instead of branching around each other
+            const float p = fast_exp2(fmaf(s, P.scale_log2, tok[i] >= 0 ? nl2 : -CUDART_INF_F)); // nl2 = -inf: p = 0
+            const float ds = p * (dp + nd);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+                dq[e] = fmaf(ds, k.v[e], dq[e]);
+                dk[i][e] = fmaf(ds, q.v[e], dk[i][e]);
+                dv[i][e] = fmaf(p, dO.v[e], dv[i][e]);
             }
         }
-        // the rows of the next head are requested before this head's arithmetic
-        uint4 qn = reinterpret_cast<const uint4 *>(P.Q + qoff)[sub];
-        uint4 dn = reinterpret_cast<const uint4 *>(P.dO + qoff)[sub];
-        uint4 on = make_uint4(0, 0, 0, 0);
-        float ln = 0.f; // first pass: LSE; later passes: the stored -LSE * log2(e)
-        float ndn = 0.f;
-        if (first) {
-            on = reinterpret_cast<const uint4 *>(P.O + qoff)[sub];
-            ln = P.LSE[(size_t)(g * G) * P.T + row];
-        } else { // written by lane 0 of this unit in the first pass: read past L1
-            ln = __ldcg(P.nl2 + (size_t)(g * G) * P.q_pad + r);
-            ndn = __ldcg(P.nd + (size_t)(g * G) * P.q_pad + r);
+        float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8;
+        if (FIRST) {
+            reinterpret_cast<float4 *>(dst)[0] = make_float4(dq[0] * P.scale, dq[1] * P.scale,
+                                                             dq[2] * P.scale, dq[3] * P.scale);
+            reinterpret_cast<float4 *>(dst)[1] = make_float4(dq[4] * P.scale, dq[5] * P.scale,
+                                                             dq[6] * P.scale, dq[7] * P.scale);
+        } else {
+            red_chunk(dst, dq, P.scale);
         }
-        for (int hh = 0; hh < G; ++hh) {
-            const int h = g * G + hh;
-            const float lcur = ln;
-            float nd = ndn;
-            const Chunk q = unpack_chunk(qn);
-            const Chunk dO = unpack_chunk(dn);
-            const Chunk o = unpack_chunk(on);
-            if (hh + 1 < G) {
-                qn = reinterpret_cast<const uint4 *>(P.Q + qoff + (size_t)(hh + 1) * 64)[sub];
-                dn = reinterpret_cast<const uint4 *>(P.dO + qoff + (size_t)(hh + 1) * 64)[sub];
-                if (first) {
-                    on = reinterpret_cast<const uint4 *>(P.O + qoff + (size_t)(hh + 1) * 64)[sub];
-                    ln = P.LSE[(size_t)(h + 1) * P.T + row];
-                } else {
-                    ln = __ldcg(P.nl2 + (size_t)(h + 1) * P.q_pad + r);
-                    ndn = __ldcg(P.nd + (size_t)(h + 1) * P.q_pad + r);
-                }
-            }
-            float nl2 = lcur;
-            if (first) {
-                float delta = 0.f;
+    }
 #pragma unroll
-                for (int e = 0; e < 8; ++e)
-                    delta = fmaf(dO.v[e], o.v[e], delta);
-#pragma unroll
-                for (int s = 1; s < 8; s <<= 1)
-                    delta += __shfl_xor_sync(um, delta, s);
-                nd = -delta;
-                nl2 = lcur == -CUDART_INF_F ? -CUDART_INF_F : -lcur * 1.4426950408889634f;
-                if (sub == 0) {
-                    P.nl2[(size_t)h * P.q_pad + r] = nl2;
-                    P.nd[(size_t)h * P.q_pad + r] = nd;
-                }
-            }
-            float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int i = 0; i < KEYS; ++i) {
-                const Chunk k = unpack_chunk(kp[i]);
-                const Chunk v = unpack_chunk(vp[i]);
-                float s = 0.f, dp = 0.f;
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    s = fmaf(q.v[e], k.v[e], s);
-                    dp = fmaf(dO.v[e], v.v[e], dp);
-                }
-#pragma unroll
-                for (int o2 = 1; o2 < 8; o2 <<= 1) {
-                    s += __shfl_xor_sync(um, s, o2);
-                    dp += __shfl_xor_sync(um, dp, o2);
-                }
-                // an absent key takes part with weight zero, so that the keys' chains of dependent
-                // instructions interleave instead of branching around each other
-                const float p = fast_exp2(fmaf(s, P.scale_log2, tok[i] >= 0 ? nl2 : -CUDART_INF_F)); // nl2 = -inf: p = 0
-                const float ds = p * (dp + nd);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    dq[e] = fmaf(ds, k.v[e], dq[e]);
-                    dk[i][e] = fmaf(ds, q.v[e], dk[i][e]);
-                    dv[i][e] = fmaf(p, dO.v[e], dv[i][e]);
-                }
-            }
-            float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8;
-            if (first) {
-                reinterpret_cast<float4 *>(dst)[0] = make_float4(dq[0] * P.scale, dq[1] * P.scale,
-                                                                 dq[2] * P.scale, dq[3] * P.scale);
-                reinterpret_cast<float4 *>(dst)[1] = make_float4(dq[4] * P.scale, dq[5] * P.scale,
-                                                                 dq[6] * P.scale, dq[7] * P.scale);
-            } else {
-                red_chunk(dst, dq, P.scale);
-            }
+    for (int i = 0; i < KEYS; ++i)
+        if (tok[i] >= 0) {
+            const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64 + sub * 8;
+            red_chunk(P.dK_acc + kr, dk[i], P.scale);
+            red_chunk(P.dV_acc + kr, dv[i], 1.f);
         }
-#pragma unroll
-        for (int i = 0; i < KEYS; ++i)
-            if (tok[i] >= 0) {
-                const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64 + sub * 8;
-                red_chunk(P.dK_acc + kr, dk[i], P.scale);
-                red_chunk(P.dV_acc + kr, dv[i], 1.f);
-            }
 }
 
-// Two keys per pass and four resident blocks per SM (128 registers): the kernel is bound by the
-// latency of its dependent chains (dot product, three shuffles, exp2), so more warps pay more
-// than fewer passes; four keys per pass at two blocks per SM was 20 % slower.
+// Two keys per pass and 128 registers: the arithmetic is bound by the latency of its dependent
+// chains (dot product, three shuffles, exp2), so more resident warps pay more than fewer passes.
+// Shared memory: [3][RB][Hq * 64] bf16 rows of Q, dO, O, then [2][RB][Hq] fp32 row values.
 __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
 {
     constexpr int KEYS = 2;
+    extern __shared__ __align__(128) uint8_t smem[];
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    const int RB = P.rows_per_block;
+    const int row_elems = P.Hq * 64;
+    __nv_bfloat16 *sQ = reinterpret_cast<__nv_bfloat16 *>(smem);
+    __nv_bfloat16 *sdO = sQ + (size_t)RB * row_elems;
+    __nv_bfloat16 *sO = sdO + (size_t)RB * row_elems;
+    float *snl2 = reinterpret_cast<float *>(sO + (size_t)RB * row_elems);
+    float *snd = snl2 + RB * P.Hq;
+    const int r0 = blockIdx.x * RB;
+    const int n_real = max(0, min(RB, (P.q_end - P.q_begin) - r0)); // rows of the partition
+    const uint32_t bar_a = smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar_a, 1);
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && n_real > 0) {
+        const uint32_t bytes = (uint32_t)(n_real * row_elems * 2);
+        mbar_arrive_expect_tx(bar_a, 3 * bytes);
+        const size_t off = (size_t)(P.q_begin + r0) * row_elems;
+        bulk_load(smem_u32(sQ), P.Q + off, bytes, bar_a);
+        bulk_load(smem_u32(sdO), P.dO + off, bytes, bar_a);
+        bulk_load(smem_u32(sO), P.O + off, bytes, bar_a);
+    }
+    for (int i = threadIdx.x; i < n_real * P.Hq; i += blockDim.x)
+        snl2[i] = P.LSE[(size_t)(i % P.Hq) * P.T + P.q_begin + r0 + i / P.Hq];
+    __syncthreads();
+
     const int sub = threadIdx.x & 7;
     const unsigned um = 0xffu << (threadIdx.x & 24); // the lanes of this unit
-    const size_t unit = (size_t)blockIdx.x * 16 + (threadIdx.x >> 3);
-    const int r = (int)(unit / P.Hkv), g = (int)(unit % P.Hkv);
-    if (r >= P.q_pad)
-        return; // the 8 lanes of a unit leave together
-    const int row = P.q_begin + r;
+    const int unit = threadIdx.x >> 3;
+    const int rl = unit / P.Hkv, g = unit % P.Hkv;
+    const int r = r0 + rl;
     const int G = P.Hq / P.Hkv;
-    if (row >= P.q_end) { // padded row: seen by nobody
+    const bool real = rl < n_real;
+    if (rl < RB && r < P.q_pad && !real) { // padded row: seen by nobody
         if (sub == 0) {
             for (int hh = 0; hh < G; ++hh) {
                 P.nl2[(size_t)(g * G + hh) * P.q_pad + r] = -CUDART_INF_F;
@@ -228,19 +250,31 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
             if (g == 0)
                 P.mqp[r] = META_NONE_Q;
         }
+    }
+    if (n_real == 0)
+        return;
+    // every thread waits for the rows (bounded); the units of padded rows then leave
+    if (!mbar_wait(bar_a, 0, &abort_flag)) {
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
         return;
     }
+    if (!real)
+        return; // the 8 lanes of a unit leave together
+    const int row = P.q_begin + r;
     if (g == 0 && sub == 0) {
         const int32_t mq = P.meta[row];
         P.mqp[r] = mq == META_NONE_K ? META_NONE_Q : mq;
     }
     const int qt = r / BM, rr = r % BM;
     const int ns = min(P.scount[qt], MAX_SINGLE);
-    const size_t qoff = ((size_t)row * P.Hq + (size_t)g * G) * 64;
-    single_pass<true, KEYS>(P, 0, ns, sub, um, r, g, row, qt, rr, G, qoff);
+    const __nv_bfloat16 *sq = sQ + (size_t)rl * row_elems, *sdo = sdO + (size_t)rl * row_elems,
+                        *so = sO + (size_t)rl * row_elems;
+    float *rnl2 = snl2 + rl * P.Hq, *rnd = snd + rl * P.Hq;
+    single_pass<true, KEYS>(P, 0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
     for (int i0 = KEYS; i0 < ns; i0 += KEYS) {
         __syncwarp(um); // lane 0's row values are visible to the unit's later passes
-        single_pass<false, KEYS>(P, i0, ns, sub, um, r, g, row, qt, rr, G, qoff);
+        single_pass<false, KEYS>(P, i0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
     }
 }
 
@@ -274,8 +308,25 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.T = p.T;
     P.scale = a.scale;
     P.scale_log2 = a.scale * 1.4426950408889634f;
-    const size_t units = (size_t)P.q_pad * a.Hkv; // of 8 lanes each
-    single_bwd<<<(unsigned)((units + 15) / 16), 128, 0, s>>>(P);
+    P.status = p.status;
+    // rows per block: about 16 units of 8 lanes, within the shared memory of four blocks per SM
+    const size_t row_bytes = (size_t)a.Hq * (3 * 64 * 2 + 8);
+    int rb = std::max(1, 16 / a.Hkv);
+    while (rb > 1 && rb * row_bytes > 48 * 1024)
+        --rb;
+    const size_t smem = rb * row_bytes;
+    const int threads = rb * a.Hkv * 8;
+    if (threads > 128 || smem > 200 * 1024)
+        return PEAGLE_ERR_BAD_SHAPE;
+    P.rows_per_block = rb;
+    static size_t smem_set = 0;
+    if (smem > smem_set) {
+        if (cudaFuncSetAttribute(single_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)smem) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        smem_set = smem;
+    }
+    single_bwd<<<(unsigned)((P.q_pad + rb - 1) / rb), threads, smem, s>>>(P);
     return 1;
 }
 
