@@ -309,7 +309,8 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.scale = a.scale;
     P.scale_log2 = a.scale * 1.4426950408889634f;
     P.status = p.status;
-    // rows per block: about 16 units of 8 lanes, within the shared memory of four blocks per SM
+    // rows per block: up to 16 units of 8 lanes within 48 KB of shared memory (the headline shape,
+    // 64 heads: one row, 25 KB, 64 threads; two rows per block measured the same)
     const size_t row_bytes = (size_t)a.Hq * (3 * 64 * 2 + 8);
     int rb = std::max(1, 16 / a.Hkv);
     while (rb > 1 && rb * row_bytes > 48 * 1024)

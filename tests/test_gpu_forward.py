@@ -46,6 +46,8 @@ SMALL = [
     # COD-subsampled metadata (retention 0.7): ragged depth blocks, chain tiles that are no
     # diagonals, Algorithm 1 on nested position sets
     inputs.Workload("cod_segments", (700,), 6, 4, 2, 64, n_segments=2, seed=15, cod_r=0.7),
+    # more KV heads than the pair-by-pair kernels take: chain tiles stay on the tensor-core path
+    inputs.Workload("many_kv_heads", (200,), 4, 24, 24, 64, seed=16),
 ]
 
 
