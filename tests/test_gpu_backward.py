@@ -237,9 +237,20 @@ def test_longtail_varlen_batch(ctx):
     full_size_checks(case, n_rows=3, n_keys=3)
 
 
-def test_host_entry_point_matches_device_entry_point(ctx):
-    w = inputs.Workload("host", (333,), 4, 4, 2, 64, n_segments=3, seed=4)
-    case = DeviceCase(w)
+@pytest.mark.parametrize("w,shuffle", [
+    (inputs.Workload("host", (333,), 4, 4, 2, 64, n_segments=3, seed=4), False),
+    # several 2,048-row slices per partition, two sequences
+    (inputs.Workload("host_slices", (1500, 700), 4, 4, 2, 64, n_segments=2, seed=5), False),
+    # a token order in which keys sit after their queries, several slices
+    (inputs.Workload("host_shuffled", (1300,), 4, 4, 2, 64, seed=6), True),
+], ids=["one_slice", "many_slices", "shuffled"])
+def test_host_entry_point_matches_device_entry_point(ctx, w, shuffle):
+    if shuffle:
+        cu, anchor, depth, parts = inputs.build_case(w, binding.peagle_assign_segments)
+        perm = np.random.default_rng(7).permutation(anchor.shape[0])
+        case = DeviceCase(w, anchor=anchor[perm], depth=depth[perm], cu=cu, parts=parts)
+    else:
+        case = DeviceCase(w)
     run_partitioned(ctx, case)
     hp = binding.Problem(case.cu, case.anchor, case.depth, w.K, w.n_q_heads, w.n_kv_heads,
                          w.head_dim, w.scale)
