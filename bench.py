@@ -178,6 +178,23 @@ def run_reference(args, w):
 
 
 # ------------------------------------------------------------------ CUDA arm
+def max_over_ranks(x: float, world: int, device) -> float:
+    """The slowest rank's figure (all-reduce MAX over the process group); x itself on one rank."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_value(world: int, flops_per_replica: float, ms_step: float) -> float:
+    """Whole-job useful TFLOP/s of `world` independent replicas that all finish within ms_step."""
+    return world * flops_per_replica / (ms_step * 1e-3) / 1e12
+
+
 def run_cuda(args, w):
     import torch
     import torch.distributed as dist
@@ -236,13 +253,10 @@ def run_cuda(args, w):
     launches = binding.peagle_launch_count(ctx) - launches0
     if binding.peagle_poll_status(ctx) != 0:
         raise RuntimeError("device-side error during the timed region")
-    if world > 1:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     f_fwd, f_bwd = useful_flops(w)
-    value = world * (f_fwd + f_bwd) / (ms_step * 1e-3) / 1e12
+    value = replicas_value(world, f_fwd + f_bwd, ms_step)
 
     # ---- end to end through the host entry point (pinned host buffers, copies timed)
     hQ, hK, hV, hdO = (t.pin_memory() for t in (Qc, Kc, Vc, dOc))
@@ -262,10 +276,7 @@ def run_cuda(args, w):
         host_step()
     torch.cuda.synchronize()
     e2e_s = (time.perf_counter() - t0) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(e2e_s, world, dev)
     nbytes = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))  # noqa: E731
     h2d = nbytes(hQ, hK, hV, hdO) + 2 * anchor.nbytes
     d2h = nbytes(hO, hLSE, hdQ, hdK, hdV)
