@@ -749,6 +749,11 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 const bool was_last = wk.last();
                 wk.next();
+                // the next step's Q / dO tiles start towards L2 one step before their stage is free
+                if (wk.valid && lane == 0) {
+                    tma_prefetch_3d(&tmQ, 0, wk.head(), P.q_begin + wk.qt() * BM);
+                    tma_prefetch_3d(&tmdO, 0, wk.head(), P.q_begin + wk.qt() * BM);
+                }
                 if (was_last && wk.valid)
                     ok = load_kv(wk.w, wk.kt, wk.g); // next item's K / V into the other stage
             }
@@ -839,12 +844,12 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     for (int k = 0; k < 8; ++k)
                         mma_ts_lo(tmem + C::TM_DK, tmem + C::TM_DP + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + k * 128, IDESC_KV, !first || k > 0);
+                    tc_commit(BAR(B_QEMPTY + st)); // dQ reads neither Q nor dO
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
                         mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, kv_m + kvo + k * 128, IDESC_DQ,
                                   k > 0);
                     tc_commit(BAR(B_DQFULL));
-                    tc_commit(BAR(B_QEMPTY + st));
                     if (last)
                         tc_commit(BAR(B_KVEMPTY + ks));
                     else {
