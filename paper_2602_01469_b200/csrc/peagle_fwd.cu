@@ -10,6 +10,8 @@
 //   warps 0-3  softmax of tile A (one query row per thread; online softmax in the log2 domain,
 //              log-sum-exp bookkeeping, final normalisation and store)
 //   warps 4-7  softmax of tile B
+//              (head_dim 64: the normalised O tile goes to shared memory and leaves by one tiled
+//              store per tile instead of 32 scattered 16-byte pieces per store instruction)
 //   warp  8    allocates tensor memory; lane 0 issues the MMAs of tile A
 //   warp  10   lane 0 issues the MMAs of tile B
 //   warp  9    producer: draws the items; TMA loads of Q per item and of the K / V tiles
@@ -80,7 +82,12 @@ struct FwdCfg {
     static constexpr int OFF_Q = 0;
     static constexpr int OFF_K = 2 * TILE_BYTES;
     static constexpr int OFF_V = OFF_K + NS * TILE_BYTES;
-    static constexpr int OFF_META = OFF_V + NS * TILE_BYTES;
+    // head_dim 64: the finished O tiles leave through shared memory and a tiled store (a thread
+    // that writes its own row puts 32 separate 16-byte pieces into every store instruction of its
+    // warp); head_dim 128 has no room for the two staging tiles and stores its rows directly
+    static constexpr bool O_STAGED = (D == 64);
+    static constexpr int OFF_OST = OFF_V + NS * TILE_BYTES;
+    static constexpr int OFF_META = OFF_OST + (O_STAGED ? 2 * TILE_BYTES : 0);
     static constexpr int OFF_BAR = OFF_META + NS * BN * 4;
     static constexpr int N_BAR = 1 + 4 * NS + 8 + 9;
     static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8; // tmem slot, abort flag, item queue
@@ -98,7 +105,8 @@ struct FwdCfg {
 template <int D>
 __global__ void __launch_bounds__(384, 1)
 fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-           const __grid_constant__ CUtensorMap tmV, const FwdParams P)
+           const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+           const FwdParams P)
 {
     using C = FwdCfg<D>;
     constexpr int NS = C::NS;
@@ -646,12 +654,50 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     dst[i] = z;
                 P.LSE[(size_t)h * P.T + row] = -CUDART_INF_F;
             }
-        } else if (__all_sync(0xffffffffu,
-                              ok && (cnt == 0 ||
-                                     mbar_wait(BAR(B_PVDONE + x), (t + cnt - 1) & 1, abort_flag)))) {
+        } else if ([&] {
+                       bool fin = __all_sync(0xffffffffu,
+                                             ok && (cnt == 0 || mbar_wait(BAR(B_PVDONE + x),
+                                                                          (t + cnt - 1) & 1, abort_flag)));
+                       if constexpr (C::O_STAGED) {
+                           // the four warps of the tile go on together (they meet at a barrier
+                           // below); before that, the staging tile of the previous item must
+                           // have left shared memory
+                           if (r == 0)
+                               bulk_wait_group_read<0>();
+                           fin = bar_and(1 + x, 128, fin);
+                       }
+                       return fin;
+                   }()) {
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
+            if constexpr (C::O_STAGED) {
+                // rows -> swizzled bf16 tile in shared memory -> one tiled store; the map ends at
+                // the partition's last row, so rows past it are not written
+                uint8_t *orow = sp + C::OFF_OST + x * C::TILE_BYTES + r * 128;
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint32_t o[32];
+                    tmem_ld32(tO + c * 32, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        uint4 v;
+                        v.x = pack_bf16x2(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
+                        v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
+                        v.z = pack_bf16x2(__uint_as_float(o[i + 4]) * inv, __uint_as_float(o[i + 5]) * inv);
+                        v.w = pack_bf16x2(__uint_as_float(o[i + 6]) * inv, __uint_as_float(o[i + 7]) * inv);
+                        const int j = c * 4 + (i >> 3); // 16-byte chunk of the row
+                        *reinterpret_cast<uint4 *>(orow + ((j ^ (r & 7)) << 4)) = v;
+                    }
+                }
+                fence_proxy_async_smem();
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + x) : "memory");
+                if (r == 0) {
+                    tma_store_3d(&tmO, sb + C::OFF_OST + x * C::TILE_BYTES, 0, h, it.row0);
+                    bulk_commit_group();
+                }
+            } else
 #pragma unroll
             for (int c = 0; c < D / 32; ++c) {
                 uint32_t o[32];
@@ -681,6 +727,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     }
 
     // ------------------------------------------------------------ teardown
+    if (C::O_STAGED && warp < 8 && (threadIdx.x & 127) == 0)
+        bulk_wait_group<0>(); // this thread's tile stores are complete
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
@@ -721,9 +769,10 @@ template <int D>
 static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int n_sm,
                         cudaStream_t s, cudaEvent_t ev0, cudaEvent_t ev1)
 {
-    CUtensorMap tmQ, tmK, tmV;
+    // the O map ends at the partition's last row: a tiled store does not write past it
+    CUtensorMap tmQ, tmK, tmV, tmO;
     if (make_map(enc, &tmQ, a.Q, D, a.Hq, p.T) || make_map(enc, &tmK, a.K, D, a.Hkv, p.T) ||
-        make_map(enc, &tmV, a.V, D, a.Hkv, p.T))
+        make_map(enc, &tmV, a.V, D, a.Hkv, p.T) || make_map(enc, &tmO, a.O, D, a.Hq, p.q_end))
         return PEAGLE_ERR_CUDA;
     FwdParams P;
     P.klist = p.klist;
@@ -759,7 +808,7 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int 
     P.n_items = p.n_qt * n_hb;
     if (ev0)
         cudaEventRecord(ev0, s);
-    fwd_kernel<D><<<std::min(P.n_items, n_sm), 384, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, P);
+    fwd_kernel<D><<<std::min(P.n_items, n_sm), 384, FwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmK, tmV, tmO, P);
     if (ev1)
         cudaEventRecord(ev1, s);
     return 1;
