@@ -985,9 +985,6 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (!ok)
                     break;
             }
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = dsv[j];
             {
                 // the same dS^T also goes over this group's dP^T columns: operand of dK
                 uint32_t pk[32];
@@ -1000,6 +997,9 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
                 tmem_st32(tDP, pk);
             }
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = dsv[j];
             tmem_wait_st();
             fence_proxy_async_smem();
             tc_fence_before();
