@@ -30,7 +30,7 @@ METRIC = "masked-attn fwd+bwd useful TFLOP/s"
 UNIT = "TFLOP/s"
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = {"gptoss_n4096": 2942594560 + 1447962624}
+NCU_TRAFFIC_BYTES = {"gptoss_n4096": 2941180160 + 1445631744}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
