@@ -28,9 +28,12 @@ from paper_2602_01469_b200 import inputs  # noqa: E402
 
 METRIC = "masked-attn fwd+bwd useful TFLOP/s"
 UNIT = "TFLOP/s"
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (set back to None whenever that kernel changes).
-NCU_TRAFFIC_BYTES = {"gptoss_n4096": 2941180160 + 1445631744}
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel come from
+# profiles/traffic.json, which records next to each figure the SHA-256 of the kernel's source
+# files at the time of the ncu capture; a figure whose sources have changed since reads as null.
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
+CSRC = os.path.join(ROOT, "paper_2602_01469_b200", "csrc")
+BWD_KERNEL = {64: "bwd64_kernel", 128: "bwd_kernel<128>"}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 
@@ -54,6 +57,39 @@ def useful_flops(w: inputs.Workload):
     fwd = 4 * p * w.head_dim * w.n_q_heads
     bwd = 10 * p * w.head_dim * w.n_q_heads
     return fwd, bwd
+
+
+def source_hash(files) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for name in sorted(files):
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def ncu_traffic(workload: str, kernel: str):
+    """DRAM bytes per launch of `kernel` on `workload` from the recorded ncu capture, or None when
+    there is no record or the kernel's sources are no longer the ones that were profiled."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            rec = json.load(f).get(workload, {}).get(kernel)
+        if rec and source_hash(rec["sources"]) == rec["sources_sha256"]:
+            return int(rec["dram_bytes_per_launch"])
+    except (OSError, ValueError, KeyError):
+        pass
+    return None
+
+
+def config_dict(w: inputs.Workload, T: int, n_parts: int) -> dict:
+    """The workload description both arms print."""
+    f_fwd, f_bwd = useful_flops(w)
+    return {"workload": w.name, "seq_lens": list(w.seq_lens) if len(w.seq_lens) < 4 else
+            f"{len(w.seq_lens)} sequences", "K": w.K, "total_tokens": T,
+            "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
+            "partitions": n_parts, "allowed_pairs": allowed_pairs(w),
+            "useful_tflop_per_step": (f_fwd + f_bwd) / 1e12,
+            "l2": "inputs (>1 GB) larger than L2, no flush", "parallelism": "replicas"}
 
 
 def load_peaks():
@@ -156,6 +192,14 @@ def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
+    from oracle import partition as opart
+
+    def oracle_assign(anchor, depth, K, bounds):       # Algorithm 1 as the oracle side states it
+        P = inputs.position_sets(anchor, depth, K)
+        A, _, _ = opart.assign_segments(P, len(bounds) - 1, bounds[-1], B=bounds)
+        return np.array([A[d][a + d] for a, d in zip(anchor, depth)], np.int32)
+
+    cu, _, _, parts = inputs.build_case(w, oracle_assign)
     per_step = max(2.0, min(20.0, 90.0 / max(1, args.steps + args.warmup)))
     for _ in range(args.warmup):
         oracle_sample(w, per_step / 4)
@@ -170,8 +214,9 @@ def run_reference(args, w):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot_t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": {"workload": w.name, "note": "each step is a bounded sample "
-                                        "of query rows; the value is useful FLOPs of the sample / time"},
+        "data": "synthetic", "config": config_dict(w, int(cu[-1]), len(parts)),
+        "note": "each step is a bounded sample of query rows; the value is useful FLOPs of the "
+                "sample / time",
         "cpu_baseline": last,
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -289,9 +334,10 @@ def run_cuda(args, w):
         launches_per_step = max(n_bwd // args.steps, 1)
         achieved = (f_bwd / launches_per_step) / (bwd_ms_launch * 1e-3) / 1e12
         roofline = {
-            "kernel": "bwd64_kernel" if w.head_dim == 64 else "bwd_kernel<128>", "bound": "tensor",
+            "kernel": BWD_KERNEL[w.head_dim], "bound": "tensor",
             "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-            "traffic": NCU_TRAFFIC_BYTES.get(w.name), "traffic_unit": "bytes per launch (ncu, DRAM)",
+            "traffic": ncu_traffic(w.name, BWD_KERNEL[w.head_dim]),
+            "traffic_unit": "bytes per launch (ncu, DRAM)",
             "peak_source": f"{peak_kind} bf16_tflops (burst)",
             "ms_per_launch": bwd_ms_launch, "launches_timed": int(n_bwd),
             "fwd_kernel": {"achieved": (f_fwd / launches_per_step) / (fwd_ms_launch * 1e-3) / 1e12,
@@ -304,12 +350,7 @@ def run_cuda(args, w):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "seq_lens": list(w.seq_lens) if len(w.seq_lens) < 4 else
-                       f"{len(w.seq_lens)} sequences", "K": w.K, "total_tokens": T,
-                       "n_q_heads": w.n_q_heads, "n_kv_heads": w.n_kv_heads, "head_dim": w.head_dim,
-                       "partitions": len(parts), "allowed_pairs": allowed_pairs(w),
-                       "useful_tflop_per_step": (f_fwd + f_bwd) / 1e12,
-                       "l2": "inputs (>1 GB) larger than L2, no flush", "parallelism": "replicas"},
+            "config": config_dict(w, T, len(parts)),
             "clocks": clocks.summary(),
             "e2e": {"value": world * (f_fwd + f_bwd) / e2e_s / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s},

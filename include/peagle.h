@@ -84,7 +84,8 @@ typedef struct peagle_partition {
     int32_t seq;             /* sequence index */
     peagle_range_t q;        /* query rows, inside sequence `seq`; empty = no-op */
     const peagle_range_t *k; /* host [nk]: visible keys, sorted disjoint non-empty ranges inside `seq` */
-    int32_t nk;              /* 0 = the whole sequence is visible */
+    int32_t nk;              /* 0 = the whole sequence is visible; at most 32 ranges, more is
+                                PEAGLE_ERR_TOO_LARGE */
 } peagle_partition_t;
 
 /* Creates a context on CUDA device `device` (sm_100 only).  Synchronous. */
@@ -117,7 +118,9 @@ int peagle_timing_read(peagle_ctx *ctx, double *ms_out, int64_t *n_out);
  * For every row q in part->q, head h (kv head g = h / (n_q_heads/n_kv_heads)) and visible
  * allowed key set A_q:   s_k = softmax_scale * <Q[q,h], K[k,g]>,
  *   LSE[h][q] = log sum_{k in A_q} exp(s_k),   O[q,h] = sum_k exp(s_k - LSE) V[k,g].
- * Writes O rows and LSE entries of the partition only.  All tensors dev.
+ * Writes O rows and LSE entries of the partition only.  All tensors dev.  The call's tile plan
+ * lives in context scratch: concurrent calls on one context from different streams race (use one
+ * context per stream).
  */
 int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partition_t *part,
                     const void *Q, const void *K, const void *V, void *O, float *LSE, void *stream);
@@ -148,7 +151,9 @@ int peagle_attn_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
  * before any stream capture begins.  Work is enqueued on `stream` and the call returns without
  * waiting.  `dev_status` (dev, may be NULL) is one int32 owned by the caller: the call clears it
  * on the stream, and a device-side error (PEAGLE_ERR_BAD_META, PEAGLE_ERR_TIMEOUT) is written
- * there; read it after synchronising the stream.
+ * there; read it after synchronising the stream.  With dev_status == NULL device-side errors are
+ * NOT reported: they go to a word inside the array that no call reads back (bad metadata then
+ * shows only as rows that see nothing).
  *
  * All calls on a device share the one array, and it keeps the previous call's contents (the
  * call re-initialises everything it reads).  Two calls whose GPU work overlaps -- different
@@ -195,7 +200,9 @@ int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
  * and the fp32 dK / dV sums are shared), so that the copy-in of Q / dO rows, the arithmetic and
  * the copy-out of O / LSE / dQ rows of different slices overlap on three internal streams.  Only
  * rows that belong to a partition are written to O, LSE and dQ.  prob->anchor / prob->depth are
- * HOST pointers for this call only.  Synchronous.  (This is the end-to-end call.)
+ * HOST pointers for this call only.  Synchronous, also on failure: an error return comes after
+ * the internal streams have drained, so nothing writes the caller's buffers afterwards (their
+ * contents are then unspecified).  (This is the end-to-end call.)
  */
 int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
                                  const peagle_partition_t *parts, int32_t nparts, const void *Q,

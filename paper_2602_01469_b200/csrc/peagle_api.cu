@@ -722,11 +722,13 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
                                  const void *K, const void *V, const void *dO, void *O, float *LSE,
                                  void *dQ, void *dK, void *dV)
 {
-    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV)
+    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV || (nparts > 0 && !parts))
         return PEAGLE_ERR_NULL;
     int rc = validate_problem(prob);
     if (rc != PEAGLE_OK)
         return rc;
+    if (nparts < 0)
+        return PEAGLE_ERR_BAD_RANGE;
     CK(cudaSetDevice(ctx->device));
     cudaStream_t s = nullptr;
     const size_t T = (size_t)prob->total_tokens;
@@ -769,6 +771,20 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
         if (!st)
             CK(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
     cudaStream_t s_in = ctx->hs[0], s_c = ctx->hs[1], s_out = ctx->hs[2];
+    // From here on copies into the caller's host buffers may be in flight: every error exit
+    // drains the three streams first, so that nothing writes O / LSE / dQ after the return.
+    auto drained = [&](int status) {
+        cudaStreamSynchronize(s_in);
+        cudaStreamSynchronize(s_c);
+        cudaStreamSynchronize(s_out);
+        return status;
+    };
+#define CKD(call)                                          \
+    do {                                                   \
+        cudaError_t e_ = (call);                           \
+        if (e_ != cudaSuccess)                             \
+            return drained(cuda_fail(ctx, e_, #call));     \
+    } while (0)
     size_t ev_next = 0;
     auto event = [&]() -> cudaEvent_t {
         if (ev_next == ctx->hev.size()) {
@@ -785,11 +801,11 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
     if (rc != PEAGLE_OK)
         return rc;
     float *dK_acc = static_cast<float *>(ctx->acc_buf.ptr), *dV_acc = dK_acc + n_kv;
-    CK(cudaMemcpyAsync(dKin, K, nkv, cudaMemcpyHostToDevice, s_in));
-    CK(cudaMemcpyAsync(dVin, V, nkv, cudaMemcpyHostToDevice, s_in));
-    CK(cudaMemcpyAsync(danchor, prob->anchor, nmeta, cudaMemcpyHostToDevice, s_in));
-    CK(cudaMemcpyAsync(ddepth, prob->depth, nmeta, cudaMemcpyHostToDevice, s_in));
-    CK(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s_c));
+    CKD(cudaMemcpyAsync(dKin, K, nkv, cudaMemcpyHostToDevice, s_in));
+    CKD(cudaMemcpyAsync(dVin, V, nkv, cudaMemcpyHostToDevice, s_in));
+    CKD(cudaMemcpyAsync(danchor, prob->anchor, nmeta, cudaMemcpyHostToDevice, s_in));
+    CKD(cudaMemcpyAsync(ddepth, prob->depth, nmeta, cudaMemcpyHostToDevice, s_in));
+    CKD(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s_c));
     peagle_problem_t dprob = *prob;
     dprob.anchor = reinterpret_cast<const int32_t *>(danchor);
     dprob.depth = reinterpret_cast<const int32_t *>(ddepth);
@@ -801,15 +817,15 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
             peagle_partition_t sl = parts[i];
             sl.q.begin = b0;
             sl.q.end = b1;
-            CK(cudaMemcpyAsync(dQin + off, static_cast<const uint8_t *>(Q) + off, len,
+            CKD(cudaMemcpyAsync(dQin + off, static_cast<const uint8_t *>(Q) + off, len,
                                cudaMemcpyHostToDevice, s_in));
-            CK(cudaMemcpyAsync(ddO + off, static_cast<const uint8_t *>(dO) + off, len,
+            CKD(cudaMemcpyAsync(ddO + off, static_cast<const uint8_t *>(dO) + off, len,
                                cudaMemcpyHostToDevice, s_in));
             cudaEvent_t e_in = event(), e_c = event();
             if (!e_in || !e_c)
-                return PEAGLE_ERR_CUDA;
-            CK(cudaEventRecord(e_in, s_in));
-            CK(cudaStreamWaitEvent(s_c, e_in, 0));
+                return drained(PEAGLE_ERR_CUDA);
+            CKD(cudaEventRecord(e_in, s_in));
+            CKD(cudaStreamWaitEvent(s_c, e_in, 0));
             Call c;
             rc = plan_call(ctx, &dprob, &sl, true, s_c, c);
             if (rc == PEAGLE_OK)
@@ -817,32 +833,31 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
             if (rc == PEAGLE_OK)
                 rc = run_bwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, ddO,
                              reinterpret_cast<float *>(dLSE), ddQ, dK_acc, dV_acc, s_c);
-            if (rc != PEAGLE_OK) {
-                cudaDeviceSynchronize();
-                return rc;
-            }
-            CK(cudaEventRecord(e_c, s_c));
-            CK(cudaStreamWaitEvent(s_out, e_c, 0));
-            CK(cudaMemcpyAsync(static_cast<uint8_t *>(O) + off, dOout + off, len, cudaMemcpyDeviceToHost, s_out));
-            CK(cudaMemcpyAsync(static_cast<uint8_t *>(dQ) + off, ddQ + off, len, cudaMemcpyDeviceToHost, s_out));
-            CK(cudaMemcpy2DAsync(LSE + b0, T * 4, reinterpret_cast<float *>(dLSE) + b0, T * 4,
+            if (rc != PEAGLE_OK)
+                return drained(rc);
+            CKD(cudaEventRecord(e_c, s_c));
+            CKD(cudaStreamWaitEvent(s_out, e_c, 0));
+            CKD(cudaMemcpyAsync(static_cast<uint8_t *>(O) + off, dOout + off, len, cudaMemcpyDeviceToHost, s_out));
+            CKD(cudaMemcpyAsync(static_cast<uint8_t *>(dQ) + off, ddQ + off, len, cudaMemcpyDeviceToHost, s_out));
+            CKD(cudaMemcpy2DAsync(LSE + b0, T * 4, reinterpret_cast<float *>(dLSE) + b0, T * 4,
                                  (size_t)(b1 - b0) * 4, (size_t)prob->n_q_heads,
                                  cudaMemcpyDeviceToHost, s_out));
         }
     }
     ctx->launches += launch_cast_grads(dK_acc, dV_acc, ddK, ddV, n_kv, s_c);
-    CK(cudaGetLastError());
+    CKD(cudaGetLastError());
     cudaEvent_t e_done = event();
     if (!e_done)
-        return PEAGLE_ERR_CUDA;
-    CK(cudaEventRecord(e_done, s_c));
-    CK(cudaStreamWaitEvent(s_out, e_done, 0));
-    CK(cudaMemcpyAsync(dK, ddK, nkv, cudaMemcpyDeviceToHost, s_out));
-    CK(cudaMemcpyAsync(dV, ddV, nkv, cudaMemcpyDeviceToHost, s_out));
-    CK(cudaStreamSynchronize(s_in));
-    CK(cudaStreamSynchronize(s_c));
-    CK(cudaStreamSynchronize(s_out));
+        return drained(PEAGLE_ERR_CUDA);
+    CKD(cudaEventRecord(e_done, s_c));
+    CKD(cudaStreamWaitEvent(s_out, e_done, 0));
+    CKD(cudaMemcpyAsync(dK, ddK, nkv, cudaMemcpyDeviceToHost, s_out));
+    CKD(cudaMemcpyAsync(dV, ddV, nkv, cudaMemcpyDeviceToHost, s_out));
+    CKD(cudaStreamSynchronize(s_in));
+    CKD(cudaStreamSynchronize(s_c));
+    CKD(cudaStreamSynchronize(s_out));
     return PEAGLE_OK;
+#undef CKD
 }
 
 int peagle_assign_segments(const int32_t *anchor, const int32_t *depth, int32_t count, int32_t K,

@@ -1142,6 +1142,8 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
     const size_t n_prep_pad = (size_t)q_pad * a.Hq * (D / 8);
     // Per-row values and the initial dQ staging: with SINGLE tiles, their backward does both.
     int launches = launch_bwd_single(p, a, s);
+    if (launches < 0)
+        return launches;
     if (launches == 0) {
         bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
             static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.LSE,
@@ -1171,8 +1173,7 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         P.Hkv = a.Hkv;
         P.scale = a.scale;
         P.scale_log2 = a.scale * 1.4426950408889634f;
-        static bool attr_set = false;
-        if (!attr_set) {
+        {   // per device, so set before every launch (host time only)
             const cudaError_t e =
                 (D == 64) ? cudaFuncSetAttribute(bwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Bwd64Cfg::SMEM_BYTES)
@@ -1180,7 +1181,6 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
                                                  BwdCfg<D>::SMEM_BYTES);
             if (e != cudaSuccess)
                 return PEAGLE_ERR_CUDA;
-            attr_set = true;
         }
         if (ev0)
             cudaEventRecord(ev0, s);

@@ -797,13 +797,11 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int 
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 FwdCfg<D>::SMEM_BYTES) != cudaSuccess)
-            return PEAGLE_ERR_CUDA;
-        attr_set = true;
-    }
+    // the attribute belongs to the current device's copy of the function: set before every launch
+    // (host time only), so that a process that drives several GPUs gets it on each of them
+    if (cudaFuncSetAttribute(fwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             FwdCfg<D>::SMEM_BYTES) != cudaSuccess)
+        return PEAGLE_ERR_CUDA;
     const int n_hb = P.two ? a.Hq / 2 : a.Hq;
     P.n_items = p.n_qt * n_hb;
     if (ev0)

@@ -320,13 +320,10 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     if (threads > 128 || smem > 200 * 1024)
         return PEAGLE_ERR_BAD_SHAPE;
     P.rows_per_block = rb;
-    static size_t smem_set = 0;
-    if (smem > smem_set) {
-        if (cudaFuncSetAttribute(single_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)smem) != cudaSuccess)
-            return PEAGLE_ERR_CUDA;
-        smem_set = smem;
-    }
+    // per device, so set before every launch (host time only)
+    if (cudaFuncSetAttribute(single_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+        return PEAGLE_ERR_CUDA;
     single_bwd<<<(unsigned)((P.q_pad + rb - 1) / rb), threads, smem, s>>>(P);
     return 1;
 }

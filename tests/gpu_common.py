@@ -79,3 +79,19 @@ def check_forward(got_O, got_LSE, want_O, want_LSE):
     assert np.abs(got_LSE[finite] - want_LSE[finite]).max() <= TOL_MAXABS_O
     assert rel_l2(got_O, want_O) <= TOL_RELL2_O
     assert rel_l2(got_LSE[finite], want_LSE[finite]) <= TOL_RELL2_O
+
+
+def check_rows(name, got, want, tol=TOL_RELL2_GRAD):
+    """Per-row bound beside the whole-tensor norm: every row (first axis) has relative L2 error
+    <= tol, or -- for rows whose true value is close to zero -- a largest error <= tol times the
+    largest magnitude of the whole tensor.  A handful of wrong rows among thousands passes a
+    whole-tensor norm; it does not pass this."""
+    got = np.asarray(got, np.float64).reshape(got.shape[0], -1)
+    want = np.asarray(want, np.float64).reshape(want.shape[0], -1)
+    assert np.isfinite(got).all(), name
+    err = np.linalg.norm(got - want, axis=1)
+    ref = np.linalg.norm(want, axis=1)
+    floor = tol * np.abs(want).max()
+    bad = (err > tol * ref) & (np.abs(got - want).max(axis=1) > floor)
+    assert not bad.any(), (name, int(bad.sum()), np.nonzero(bad)[0][:8].tolist(),
+                           float((err / np.maximum(ref, 1e-300))[bad].max()))

@@ -4,7 +4,7 @@ import pytest
 import torch
 
 from paper_2602_01469_b200 import binding, inputs
-from tests.gpu_common import TOL_RELL2_GRAD, DeviceCase, check_forward, rel_l2
+from tests.gpu_common import TOL_RELL2_GRAD, DeviceCase, check_forward, check_rows, rel_l2
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +47,7 @@ def check_grads(case, dQ, dK, dV):
     for name, g, want in zip(("dQ", "dK", "dV"), got, (dQ, dK, dV)):
         assert np.isfinite(g).all(), name
         assert rel_l2(g, want) <= TOL_RELL2_GRAD, (name, rel_l2(g, want))
+        check_rows(name, g, want)
 
 
 SMALL = [
@@ -165,6 +166,7 @@ def full_size_checks(case, n_rows=16, n_keys=6, seed=0):
         dQ, _, _ = case.oracle_bwd(p, rows=rows)
         g = got_dQ[torch.as_tensor(rows, device="cuda")].cpu().numpy()
         assert rel_l2(g, dQ) <= TOL_RELL2_GRAD
+        check_rows("dQ", g, dQ)
     # (4) dK / dV of keys few queries see: chain tokens (depth >= 1) and the last depth-0
     # tokens of a sequence; every query that sees them is evaluated by the oracle
     for s in range(len(case.cu) - 1):
@@ -191,6 +193,8 @@ def full_size_checks(case, n_rows=16, n_keys=6, seed=0):
         kt = torch.as_tensor(keys + sl.start, device="cuda")
         assert rel_l2(got_dK[kt].cpu().numpy(), dKs[keys]) <= TOL_RELL2_GRAD
         assert rel_l2(got_dV[kt].cpu().numpy(), dVs[keys]) <= TOL_RELL2_GRAD
+        check_rows("dK", got_dK[kt].cpu().numpy(), dKs[keys])
+        check_rows("dV", got_dV[kt].cpu().numpy(), dVs[keys])
         if s >= 2:
             break
 
@@ -216,6 +220,32 @@ def test_partitioned_one_kv_group_in_full(ctx):
     assert rel_l2(case.dQ[:, :G].float().cpu().numpy(), dQ) <= TOL_RELL2_GRAD
     assert rel_l2(case.dK[:, 0].float().cpu().numpy(), dK[:, 0]) <= TOL_RELL2_GRAD
     assert rel_l2(case.dV[:, 0].float().cpu().numpy(), dV[:, 0]) <= TOL_RELL2_GRAD
+    check_rows("dQ", case.dQ[:, :G].float().cpu().numpy(), dQ)
+    check_rows("dK", case.dK[:, 0].float().cpu().numpy(), dK[:, 0])
+    check_rows("dV", case.dV[:, 0].float().cpu().numpy(), dV[:, 0])
+
+
+def test_headline_one_kv_group_in_full(ctx):
+    """Config 3 (the headline shape) restricted to one KV group: O, LSE, dQ of its 8 query heads
+    and dK, dV of the group, every row, whole-tensor norms and per-row bounds.  This is the path
+    that only exists at full size: every early depth-0 key row is the sum of reductions from
+    hundreds of work items."""
+    w = inputs.WORKLOADS["gptoss_n4096"]
+    case = DeviceCase(w)
+    run_partitioned(ctx, case)
+    G = w.n_q_heads // w.n_kv_heads
+    g = 3
+    hs = (g * G, (g + 1) * G)
+    p = case.parts[0]
+    O, LSE = case.oracle_fwd(p, heads=hs)
+    dQ, dK, dV = case.oracle_bwd(p, heads=hs)
+    check_forward(case.O[:, hs[0]:hs[1]].float().cpu().numpy(),
+                  case.LSE[hs[0]:hs[1]].t().cpu().numpy(), O, LSE)
+    got = {"dQ": case.dQ[:, hs[0]:hs[1]].float().cpu().numpy(),
+           "dK": case.dK[:, g].float().cpu().numpy(), "dV": case.dV[:, g].float().cpu().numpy()}
+    for name, want in (("dQ", dQ), ("dK", dK[:, g]), ("dV", dV[:, g])):
+        assert rel_l2(got[name], want) <= TOL_RELL2_GRAD, name
+        check_rows(name, got[name], want)
 
 
 def test_longtail_varlen_batch(ctx):
@@ -235,6 +265,16 @@ def test_longtail_varlen_batch(ctx):
     assert rel_l2(case.dK[sl, 0].float().cpu().numpy(), dK[:, 0]) <= TOL_RELL2_GRAD
     assert rel_l2(case.dV[sl, 0].float().cpu().numpy(), dV[:, 0]) <= TOL_RELL2_GRAD
     full_size_checks(case, n_rows=3, n_keys=3)
+    # O / LSE of the two sequences that are split into two partitions, sampled rows of each part
+    rng = np.random.default_rng(1)
+    split = [q for q in case.parts if sum(1 for r in case.parts if r["seq"] == q["seq"]) > 1]
+    assert len(split) == 4
+    for p in split:
+        b, e = p["q"]
+        rows = np.unique(np.concatenate([[b, e - 1], rng.integers(b, e, size=6)]))
+        O, LSE = case.oracle_fwd(p, rows=rows)
+        rt = torch.as_tensor(rows, device="cuda")
+        check_forward(case.O[rt].float().cpu().numpy(), case.LSE[:, rt].t().cpu().numpy(), O, LSE)
 
 
 @pytest.mark.parametrize("w,shuffle", [

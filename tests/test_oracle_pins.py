@@ -384,3 +384,98 @@ def test_partitioned_equals_unpartitioned(case):
         M = orc.mask_dense(anchor, depth)
         assert not M[rows][:, ~vis].any()
     assert np.allclose(dKp, dK, atol=1e-12) and np.allclose(dVp, dV, atol=1e-12)
+
+
+# ---------------------------------------------------------------- visible key ranges
+def hidden_mask(anchor, depth, kranges):
+    """The mask with the columns outside the half-open ranges zeroed by hand."""
+    M = dense_from_sets(anchor, depth).copy()
+    vis = np.zeros(len(anchor), bool)
+    for b, e in kranges:
+        vis[b:e] = True
+    M[:, ~vis] = 0
+    return M
+
+
+def test_key_ranges_hide_part_of_the_allowed_set():
+    """A partition's visible ranges cut into rows' allowed sets: ranges that end one token before
+    and one token after an allowed key, a gap in the middle, and a range starting past token 0.
+    Forward, backward and the pair count must equal the dense formulation on a mask whose hidden
+    columns this test zeroes itself (half-open ranges: `begin` is visible, `end` is not)."""
+    n, K, Hq, Hkv, D = 10, 4, 4, 2, 8
+    anchor, depth, Q, Kt, V, dO = rand_case(n, K, Hq, Hkv, D, seed=21, std=1.0)
+    perm = np.random.default_rng(5).permutation(n * K)
+    anchor, depth = anchor[perm], depth[perm]
+    T = n * K
+    full = dense_from_sets(anchor, depth)
+    # pick a row with many allowed keys and cut right before / right after two of them
+    q_big = int(np.argmax(full.sum(1)))
+    ks = np.nonzero(full[q_big])[0]
+    k_lo, k_hi = int(ks[1]), int(ks[-2])
+    assert k_lo + 1 < k_hi
+    cases = [
+        [(0, k_lo), (k_lo + 1, k_hi + 1)],      # ends one before an allowed key; k_hi is the last visible
+        [(1, k_lo + 1), (k_hi, T)],             # ends one after it (k_lo visible); token 0 hidden
+        [(3, 17), (18, 19), (25, T - 2)],       # three ranges, one of a single token
+    ]
+    for kr in cases:
+        M = hidden_mask(anchor, depth, kr)
+        part = M.sum(1)
+        assert ((part > 0) & (part < full.sum(1))).sum() >= 5      # rows hidden only in part
+        assert orc.count_pairs(anchor, depth, kranges=kr) == int(M.sum())
+        rows = np.arange(T)
+        assert orc.count_pairs(anchor, depth, rows=rows[::3], kranges=kr) == int(M[::3].sum())
+        q = Q.double().requires_grad_()
+        k = Kt.double().requires_grad_()
+        v = V.double().requires_grad_()
+        live = torch.as_tensor(M.sum(1) > 0)
+        ref_O, ref_L = torch_dense_attention(M[live.numpy()], q[live], k, v, 0.29)
+        (ref_O * dO.double()[live]).sum().backward()
+        O, LSE = orc.attn_fwd(anchor, depth, Q, Kt, V, 0.29, kranges=kr)
+        dQ, dK, dV = orc.attn_bwd(anchor, depth, Q, Kt, V, dO, 0.29, kranges=kr)
+        lv = live.numpy()
+        assert np.allclose(O[lv], ref_O.detach().numpy(), atol=1e-12)
+        assert np.allclose(LSE[lv], ref_L.detach().numpy(), atol=1e-12)
+        assert np.all(O[~lv] == 0) and np.all(np.isneginf(LSE[~lv]))
+        assert np.allclose(dQ, q.grad.numpy(), atol=1e-11)       # rows that see nothing: zero
+        assert np.allclose(dK, k.grad.numpy(), atol=1e-11)
+        assert np.allclose(dV, v.grad.numpy(), atol=1e-11)
+        hidden = np.ones(T, bool)
+        for b, e in kr:
+            hidden[b:e] = False
+        assert np.all(dK[hidden] == 0) and np.all(dV[hidden] == 0)
+
+
+@pytest.mark.parametrize("case", ["full_grid", "fig3", "cod"])
+def test_layout_key_ranges_are_alg1_cumulative_depth0_sets(case):
+    """Algorithm 1, phase 3: segment s sees the depth-0 positions p < B[s+1].  The ranges the
+    layout helper hands to both sides must hold, outside the segment's own block, exactly the
+    depth-0 tokens of N[s] that earlier segments own -- token for token."""
+    if case == "full_grid":
+        n, K, S = 45, 5, 4
+        anchor, depth = inputs.full_grid(n, K)
+    elif case == "fig3":
+        n, K, S = 16, 4, 2
+        _, anchor, depth = fig3_tokens()
+    else:
+        n, K, S = 60, 6, 3
+        anchor, depth = inputs.cod_grid(n, K, 0.7, seed=2)
+    P = inputs.position_sets(anchor, depth, K)
+    A, N, B = opart.assign_segments(P, S, n)
+    seg = np.array([A[d][a + d] for a, d in zip(anchor, depth)], np.int32)
+    perm = inputs.arrange_by_segment(anchor, depth, seg)
+    anchor, depth, seg = anchor[perm], depth[perm], seg[perm]
+    parts = inputs.partitions_from_layout(seg, depth)
+    assert len(parts) == S
+    for s, p in enumerate(parts):
+        own = set(range(*p["q"]))
+        assert own == set(np.nonzero(seg == s)[0].tolist())
+        vis = set()
+        for b, e in p["k"]:
+            vis |= set(range(b, e))
+        assert own <= vis
+        outside = vis - own
+        assert all(depth[t] == 0 for t in outside)
+        # depth-0 positions visible to segment s, as Algorithm 1 lists them
+        vis_d0 = sorted(int(anchor[t]) for t in vis if depth[t] == 0)
+        assert vis_d0 == N[s]

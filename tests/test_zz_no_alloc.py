@@ -1,10 +1,13 @@
-"""GPU: the allocation-free forward entry point against the ordinary one, through the C ABI.
+"""GPU: the allocation-free forward entry point against the fp64 oracle, through the C ABI.
 
 ``peagle_attn_fwd_static`` is for callers that cannot call cudaMalloc (a step running inside a
 framework whose allocator owns the GPU's memory, a loop that cannot take an allocation's
 device-wide synchronisation).  Its tile plan lives in one fixed array inside the library that
-every call reuses, so the thing to check is that a call is not disturbed by what the previous
-call left there: two calls in a row on different partitions, then the first one again.
+every call reuses, so the things to check are: its results are right (against the oracle, and
+equal to the ordinary entry point's), a call is not disturbed by what the previous call left in
+the array (two calls in a row on different partitions, then the first one again), it really
+allocates nothing (free device memory is unchanged across a call), and it works at the largest
+shape it accepts.
 
 This file sorts last on purpose: a run that stops at the first failure has then already run
 every other test.
@@ -14,7 +17,7 @@ import pytest
 import torch
 
 from paper_2602_01469_b200 import binding, inputs
-from tests.gpu_common import TOL_MAXABS_O, TOL_RELL2_O, DeviceCase, rel_l2
+from tests.gpu_common import DeviceCase, check_forward
 
 pytestmark = pytest.mark.gpu
 
@@ -25,22 +28,12 @@ def fresh_outputs(case):
 
 
 def rows_of(part, O, LSE):
+    """O [rows][H][D], LSE [rows][H] of a partition's query rows."""
     b, e = part["q"]
-    return O[b:e].float().cpu().numpy(), LSE[:, b:e].cpu().numpy()
+    return O[b:e].float().cpu().numpy(), LSE[:, b:e].t().cpu().numpy()
 
 
-def assert_matches(got, want):
-    (gO, gL), (wO, wL) = got, want
-    assert np.isfinite(gO).all()
-    finite = np.isfinite(wL)
-    assert np.array_equal(np.isneginf(gL), np.isneginf(wL))
-    assert np.abs(gO - wO).max() <= TOL_MAXABS_O
-    assert np.abs(gL[finite] - wL[finite]).max() <= TOL_MAXABS_O
-    assert rel_l2(gO, wO) <= TOL_RELL2_O
-    assert rel_l2(gL[finite], wL[finite]) <= TOL_RELL2_O
-
-
-def test_static_forward_matches_context_forward_on_consecutive_calls():
+def test_static_forward_matches_oracle_and_context_forward_on_consecutive_calls():
     # three segments: partitions with one, two and three visible key ranges, ragged tiles
     w = inputs.Workload("no_alloc", (333,), 4, 4, 2, 64, n_segments=3, seed=12)
     case = DeviceCase(w)
@@ -51,19 +44,53 @@ def test_static_forward_matches_context_forward_on_consecutive_calls():
         assert binding.peagle_poll_status(ctx) == 0
     finally:
         ctx.close()
+    want = [case.oracle_fwd(p) for p in case.parts]
     status = torch.full((1,), 77, dtype=torch.int32, device="cuda:0")
     # largest partition first, then a smaller one over the leftovers, then the first again
     order = [len(case.parts) - 1, 0, len(case.parts) - 1]
-    for i in order:
+    for n_call, i in enumerate(order):
         O, LSE = fresh_outputs(case)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info(0)[0]
         binding.peagle_attn_fwd_static(0, case.prob, case.bparts[i], case.dQ_, case.dK_, case.dV_,
                                        O, LSE, status)
         torch.cuda.synchronize()
+        if n_call > 0:       # the first call on a device may load the kernels' code
+            assert torch.cuda.mem_get_info(0)[0] == free_before, "the call allocated device memory"
         assert int(status.item()) == 0
         part = case.parts[i]
-        assert_matches(rows_of(part, O, LSE), rows_of(part, case.O, case.LSE))
+        gO, gL = rows_of(part, O, LSE)
+        check_forward(gO, gL, *want[i])                       # against the fp64 oracle
+        cO, cL = rows_of(part, case.O, case.LSE)              # and the same bits as the context path
+        assert np.array_equal(gO, cO) and np.array_equal(gL, cL)
         b, e = part["q"]                      # rows outside the partition stay untouched
         assert torch.isnan(O[:b].float()).all() and torch.isnan(O[e:].float()).all()
+    # without a status word: same result (device-side errors would go unreported)
+    O, LSE = fresh_outputs(case)
+    binding.peagle_attn_fwd_static(0, case.prob, case.bparts[0], case.dQ_, case.dK_, case.dV_, O, LSE,
+                                   None)
+    torch.cuda.synchronize()
+    check_forward(*rows_of(case.parts[0], O, LSE), *want[0])
+
+
+def test_static_forward_at_its_limit_shape():
+    """The largest call it accepts: 32,768 tokens, 256 x 256 tiles (the headline grid), sampled
+    rows against the oracle."""
+    w = inputs.WORKLOADS["gptoss_n4096"]
+    case = DeviceCase(w)
+    assert case.T == 32768
+    status = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    O, LSE = fresh_outputs(case)
+    binding.peagle_attn_fwd_static(0, case.prob, case.bparts[0], case.dQ_, case.dK_, case.dV_, O, LSE,
+                                   status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    assert torch.isfinite(O.float()).all() and torch.isfinite(LSE).all()
+    rng = np.random.default_rng(2)
+    rows = np.unique(np.concatenate([[0, case.T - 1], rng.integers(0, case.T, size=24)]))
+    wO, wL = case.oracle_fwd(case.parts[0], rows=rows)
+    rt = torch.as_tensor(rows, device="cuda")
+    check_forward(O[rt].float().cpu().numpy(), LSE[:, rt].t().cpu().numpy(), wO, wL)
 
 
 def test_static_forward_rejects_sizes_beyond_its_limit():
