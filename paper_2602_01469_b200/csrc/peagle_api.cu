@@ -239,12 +239,40 @@ int plan_call(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partit
     return PEAGLE_OK;
 }
 
+// Scratch of one backward call inside ctx->bwd_buf: per-row values and the fp32 dQ staging.
+int bwd_scratch(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, cudaStream_t s,
+                BwdArgs &a)
+{
+    const size_t q_len = (size_t)(c.plan.q_end - c.plan.q_begin);
+    const size_t Hq = (size_t)prob->n_q_heads, D = (size_t)prob->head_dim;
+    const size_t q_pad = (size_t)c.plan.n_qt * BM;
+    const size_t row_bytes = ((2 * Hq + 1) * q_pad * 4 + 255) / 256 * 256;
+    const size_t dq_bytes = q_len * Hq * D * 4;
+    int rc = ensure(ctx, ctx->bwd_buf, row_bytes + dq_bytes + 256, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    a.nl2 = static_cast<float *>(ctx->bwd_buf.ptr);
+    a.nd = a.nl2 + Hq * q_pad;
+    a.mqp = reinterpret_cast<int32_t *>(a.nd + Hq * q_pad);
+    a.dq_acc = reinterpret_cast<float *>(static_cast<uint8_t *>(ctx->bwd_buf.ptr) + row_bytes);
+    return PEAGLE_OK;
+}
+
+// `hand`: when the caller already knows dO (the partition driver), the backward's row scratch
+// that the forward's epilogue fills (-LSE * log2 e, -Delta, packed metadata); else null.
 int run_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const void *Q,
-            const void *K, const void *V, void *O, float *LSE, cudaStream_t s)
+            const void *K, const void *V, void *O, float *LSE, cudaStream_t s,
+            const void *dO = nullptr, const BwdArgs *hand = nullptr)
 {
     if (c.plan.n_qt == 0)
         return PEAGLE_OK;
     FwdArgs a;
+    if (hand) {
+        a.dO = dO;
+        a.nl2 = hand->nl2;
+        a.nd = hand->nd;
+        a.mqp = hand->mqp;
+    }
     a.Q = Q;
     a.K = K;
     a.V = V;
@@ -266,19 +294,15 @@ int run_fwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
 
 int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const void *Q,
             const void *K, const void *V, const void *O, const void *dO, const float *LSE,
-            void *dQ, float *dK_acc, float *dV_acc, cudaStream_t s)
+            void *dQ, float *dK_acc, float *dV_acc, cudaStream_t s, bool rows_ready = false)
 {
     if (c.plan.n_qt == 0)
         return PEAGLE_OK;
-    const size_t q_len = (size_t)(c.plan.q_end - c.plan.q_begin);
-    const size_t Hq = (size_t)prob->n_q_heads, D = (size_t)prob->head_dim;
-    const size_t q_pad = (size_t)c.plan.n_qt * BM;
-    const size_t row_bytes = ((2 * Hq + 1) * q_pad * 4 + 255) / 256 * 256;
-    const size_t dq_bytes = q_len * Hq * D * 4;
-    int rc = ensure(ctx, ctx->bwd_buf, row_bytes + dq_bytes + 256, s);
+    BwdArgs a;
+    int rc = bwd_scratch(ctx, prob, c, s, a);
     if (rc != PEAGLE_OK)
         return rc;
-    BwdArgs a;
+    a.rows_ready = rows_ready;
     a.Q = Q;
     a.K = K;
     a.V = V;
@@ -288,10 +312,6 @@ int run_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const Call &c, const 
     a.dQ = dQ;
     a.dK_acc = dK_acc;
     a.dV_acc = dV_acc;
-    a.nl2 = static_cast<float *>(ctx->bwd_buf.ptr);
-    a.nd = a.nl2 + Hq * q_pad;
-    a.mqp = reinterpret_cast<int32_t *>(a.nd + Hq * q_pad);
-    a.dq_acc = reinterpret_cast<float *>(static_cast<uint8_t *>(ctx->bwd_buf.ptr) + row_bytes);
     a.Hq = prob->n_q_heads;
     a.Hkv = prob->n_kv_heads;
     a.D = prob->head_dim;
@@ -705,10 +725,18 @@ int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
         rc = plan_call(ctx, prob, &parts[i], true, s, c);
         if (rc != PEAGLE_OK)
             return rc;
-        rc = run_fwd(ctx, prob, c, Q, K, V, O, LSE, s);
+        // dO is known here, so the forward's epilogue leaves the backward's per-row values
+        // (the separate peagle_attn_bwd forms them itself from O, dO and LSE)
+        BwdArgs hand;
+        if (c.plan.n_qt > 0) {
+            rc = bwd_scratch(ctx, prob, c, s, hand);
+            if (rc != PEAGLE_OK)
+                return rc;
+        }
+        rc = run_fwd(ctx, prob, c, Q, K, V, O, LSE, s, dO, &hand);
         if (rc != PEAGLE_OK)
             return rc;
-        rc = run_bwd(ctx, prob, c, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc, s);
+        rc = run_bwd(ctx, prob, c, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc, s, true);
         if (rc != PEAGLE_OK)
             return rc;
     }
@@ -828,11 +856,15 @@ int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
             CKD(cudaStreamWaitEvent(s_c, e_in, 0));
             Call c;
             rc = plan_call(ctx, &dprob, &sl, true, s_c, c);
+            BwdArgs hand;
+            if (rc == PEAGLE_OK && c.plan.n_qt > 0)
+                rc = bwd_scratch(ctx, &dprob, c, s_c, hand);
             if (rc == PEAGLE_OK)
-                rc = run_fwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, reinterpret_cast<float *>(dLSE), s_c);
+                rc = run_fwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, reinterpret_cast<float *>(dLSE), s_c,
+                             ddO, &hand);
             if (rc == PEAGLE_OK)
                 rc = run_bwd(ctx, &dprob, c, dQin, dKin, dVin, dOout, ddO,
-                             reinterpret_cast<float *>(dLSE), ddQ, dK_acc, dV_acc, s_c);
+                             reinterpret_cast<float *>(dLSE), ddQ, dK_acc, dV_acc, s_c, true);
             if (rc != PEAGLE_OK)
                 return drained(rc);
             CKD(cudaEventRecord(e_c, s_c));

@@ -1144,7 +1144,11 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
     int launches = launch_bwd_single(p, a, s);
     if (launches < 0)
         return launches;
-    if (launches == 0) {
+    if (launches == 0 && a.rows_ready) {
+        // the forward of this partition left the per-row values; only the staging needs clearing
+        if (cudaMemsetAsync(a.dq_acc, 0, (size_t)q_len * a.Hq * D * sizeof(float), s) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+    } else if (launches == 0) {
         bwd_prepare<D><<<(unsigned)((n_prep_pad + 255) / 256), 256, 0, s>>>(
             static_cast<const __nv_bfloat16 *>(a.O), static_cast<const __nv_bfloat16 *>(a.dO), a.LSE,
             p.meta, a.nl2, a.nd, a.mqp, a.dq_acc, p.q_begin, q_len, q_pad, a.Hq, p.T);

@@ -54,6 +54,13 @@ struct FwdParams {
     const uint8_t *scs;  // [n_qt][MAX_SINGLE][BM] key column of entry i for row r, or NO_COL
     const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
     const __nv_bfloat16 *Q, *K, *V;
+    // Optional hand-over to the backward of the same partition (the driver knows dO when the
+    // forward runs): per (head, row) -LSE * log2(e) and -Delta = -<dO, O>, [Hq][q_pad] each, and
+    // the rows' packed metadata [q_pad], neutral values for the rows past the partition's end.
+    const __nv_bfloat16 *dO; // null: nothing is handed over
+    float *nl2, *nd;
+    int32_t *mqp;
+    int q_pad;
 };
 
 // <a, b> of two rows of 64 bf16 held as 32 packed pairs; products are exact in fp32.
@@ -167,9 +174,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         }
         for (int x = 0; x < 2; ++x) {
             mbar_init(BAR(B_SFULL + x), 1);
-            mbar_init(BAR(B_PFULL + x), 128);
+            mbar_init(BAR(B_PFULL + x), 4);   // one arrival per softmax warp of the tile
             mbar_init(BAR(B_PVDONE + x), 1);
-            mbar_init(BAR(B_SREAD + x), 128);
+            mbar_init(BAR(B_SREAD + x), 4);
         }
         for (int i = 0; i < 4; ++i) {
             mbar_init(BAR(B_WQFULL + i), 1);
@@ -442,6 +449,12 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         if (mq == META_NONE_K)
             mq = META_NONE_Q;
         float m = -CUDART_INF_F, l = 0.f;
+        if (P.dO && row_ok) { // the epilogue reads this row of dO
+            const __nv_bfloat16 *pre = P.dO + ((size_t)row * P.Hq + h) * D;
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(pre));
+            if (D == 128)
+                asm volatile("prefetch.global.L2 [%0];" ::"l"(pre + 64));
+        }
         if (n_single == 0 && lane == 0)
             mbar_arrive(BAR(B_QEMPTY)); // no row of Q is read by this warp
         if constexpr (D == 64) {
@@ -560,7 +573,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tmem_wait_ld();
             // S(j) is in registers: its columns may be overwritten by S(j+1)
             tc_fence_before();
-            mbar_arrive(BAR(B_SREAD + x));
+            warp_arrive(BAR(B_SREAD + x));
             if (cls != TILE_FULL) {
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
                 if (!ok)
@@ -643,9 +656,27 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             l += sum;
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(BAR(B_PFULL + x));
+            warp_arrive(BAR(B_PFULL + x));
         }
         // ---- epilogue: normalise, store O and LSE
+        // Delta of the row needs the row of dO: requested here, ahead of the wait for the last
+        // P V product (the row was sent towards L2 when the item began)
+        const bool want_delta = P.dO != nullptr && row_ok && (cnt > 0 || n_single > 0);
+        uint4 dov[D / 8];
+        if (want_delta) {
+            const uint4 *src = reinterpret_cast<const uint4 *>(P.dO + ((size_t)row * P.Hq + h) * D);
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i)
+                dov[i] = __ldg(src + i);
+        } else {
+#pragma unroll
+            for (int i = 0; i < D / 8; ++i)
+                dov[i] = make_uint4(0, 0, 0, 0);
+        }
+        // rows of the padded partition are numbered from its first row
+        const size_t hand = (size_t)h * P.q_pad + (size_t)(qt * BM + r);
+        if (P.dO && x == 0 && (it.h0 == 0))
+            P.mqp[qt * BM + r] = mq;
         if (cnt == 0 && n_single == 0) {
             if (row_ok) {
                 uint4 z = make_uint4(0, 0, 0, 0);
@@ -653,6 +684,10 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 for (int i = 0; i < D / 8; ++i)
                     dst[i] = z;
                 P.LSE[(size_t)h * P.T + row] = -CUDART_INF_F;
+            }
+            if (P.dO) {
+                P.nl2[hand] = -CUDART_INF_F;
+                P.nd[hand] = 0.f;
             }
         } else if ([&] {
                        bool fin = __all_sync(0xffffffffu,
@@ -671,6 +706,15 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             tc_fence_after();
             const float inv = l > 0.f ? 1.f / l : 0.f;
             uint4 *dst = reinterpret_cast<uint4 *>(P.O + ((size_t)row * P.Hq + h) * D);
+            float delta = 0.f;
+            auto dot8 = [&](const uint4 w, const uint32_t *o8) {
+                const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    delta = fmaf(__uint_as_float(ww[k] << 16), __uint_as_float(o8[2 * k]), delta);
+                    delta = fmaf(__uint_as_float(ww[k] & 0xffff0000u), __uint_as_float(o8[2 * k + 1]), delta);
+                }
+            };
             if constexpr (C::O_STAGED) {
                 // rows -> swizzled bf16 tile in shared memory -> one tiled store; the map ends at
                 // the partition's last row, so rows past it are not written
@@ -682,6 +726,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     tmem_wait_ld();
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
+                        dot8(dov[c * 4 + (i >> 3)], o + i);
                         uint4 v;
                         v.x = pack_bf16x2(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
                         v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
@@ -706,6 +751,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 if (row_ok) {
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
+                        dot8(dov[c * 4 + (i >> 3)], o + i);
                         uint4 v;
                         v.x = pack_bf16x2(__uint_as_float(o[i + 0]) * inv, __uint_as_float(o[i + 1]) * inv);
                         v.y = pack_bf16x2(__uint_as_float(o[i + 2]) * inv, __uint_as_float(o[i + 3]) * inv);
@@ -715,9 +761,13 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     }
                 }
             }
+            const float lse2 = l > 0.f ? m + log2f(l) : -CUDART_INF_F;
             if (row_ok)
-                P.LSE[(size_t)h * P.T + row] =
-                    l > 0.f ? (m + log2f(l)) * 0.6931471805599453f : -CUDART_INF_F;
+                P.LSE[(size_t)h * P.T + row] = lse2 * 0.6931471805599453f;
+            if (P.dO) { // the accumulator is not normalised: Delta = inv * <dO, O_acc>
+                P.nl2[hand] = (row_ok && l > 0.f) ? -lse2 : -CUDART_INF_F;
+                P.nd[hand] = row_ok ? -delta * inv : 0.f;
+            }
         } else {
             ok = false; // a wait ran out
         }
@@ -794,6 +844,11 @@ static int launch_fwd_t(const Plan &p, const FwdArgs &a, EncodeTiledFn enc, int 
     P.scount = p.scount;
     P.scs = p.scs;
     P.sbase = p.sbase;
+    P.dO = static_cast<const __nv_bfloat16 *>(a.dO);
+    P.nl2 = a.nl2;
+    P.nd = a.nd;
+    P.mqp = a.mqp;
+    P.q_pad = p.n_qt * BM;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);

@@ -65,6 +65,11 @@ struct FwdArgs {
     float *LSE;
     int Hq, Hkv, D;
     float scale;
+    // optional hand-over to the backward of the same partition (all null when not wanted):
+    // dO and the backward's per-row scratch, which the forward's epilogue then fills
+    const void *dO = nullptr;
+    float *nl2 = nullptr, *nd = nullptr;
+    int32_t *mqp = nullptr;
 };
 
 struct BwdArgs {
@@ -79,6 +84,7 @@ struct BwdArgs {
     float *dq_acc;  // [q_len][Hq][D] scratch, fp32
     int Hq, Hkv, D;
     float scale;
+    bool rows_ready = false; // nl2 / nd / mqp were written by the forward of this partition
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,

@@ -34,6 +34,7 @@ struct SingleParams {
     float *dq_acc, *dK_acc, *dV_acc;
     int *status;
     int q_begin, q_end, q_pad, n_qt, Hq, Hkv, T, rows_per_block;
+    int rows_ready; // 1: nl2 / nd / mqp were already written by the forward (O and LSE are not read)
     float scale, scale_log2;
 };
 
@@ -128,7 +129,10 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
         const Chunk q = load_chunk(sq + (size_t)h * 64, sub);
         const Chunk dO = load_chunk(sdo + (size_t)h * 64, sub);
         float nl2, nd;
-        if (FIRST) {
+        if (FIRST && P.rows_ready) {
+            nl2 = snl2[h];
+            nd = snd[h];
+        } else if (FIRST) {
             const Chunk o = load_chunk(so + (size_t)h * 64, sub);
             float delta = 0.f;
 #pragma unroll
@@ -224,14 +228,23 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
     __syncthreads();
     if (threadIdx.x == 0 && n_real > 0) {
         const uint32_t bytes = (uint32_t)(n_real * row_elems * 2);
-        mbar_arrive_expect_tx(bar_a, 3 * bytes);
+        mbar_arrive_expect_tx(bar_a, (P.rows_ready ? 2 : 3) * bytes);
         const size_t off = (size_t)(P.q_begin + r0) * row_elems;
         bulk_load(smem_u32(sQ), P.Q + off, bytes, bar_a);
         bulk_load(smem_u32(sdO), P.dO + off, bytes, bar_a);
-        bulk_load(smem_u32(sO), P.O + off, bytes, bar_a);
+        if (!P.rows_ready)
+            bulk_load(smem_u32(sO), P.O + off, bytes, bar_a);
     }
-    for (int i = threadIdx.x; i < n_real * P.Hq; i += blockDim.x)
-        snl2[i] = P.LSE[(size_t)(i % P.Hq) * P.T + P.q_begin + r0 + i / P.Hq];
+    if (P.rows_ready) {
+        for (int i = threadIdx.x; i < n_real * P.Hq; i += blockDim.x) {
+            const size_t ri = (size_t)(i % P.Hq) * P.q_pad + r0 + i / P.Hq;
+            snl2[i] = P.nl2[ri];
+            snd[i] = P.nd[ri];
+        }
+    } else {
+        for (int i = threadIdx.x; i < n_real * P.Hq; i += blockDim.x)
+            snl2[i] = P.LSE[(size_t)(i % P.Hq) * P.T + P.q_begin + r0 + i / P.Hq];
+    }
     __syncthreads();
 
     const int sub = threadIdx.x & 7;
@@ -241,7 +254,7 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
     const int r = r0 + rl;
     const int G = P.Hq / P.Hkv;
     const bool real = rl < n_real;
-    if (rl < RB && r < P.q_pad && !real) { // padded row: seen by nobody
+    if (rl < RB && r < P.q_pad && !real && !P.rows_ready) { // padded row: seen by nobody
         if (sub == 0) {
             for (int hh = 0; hh < G; ++hh) {
                 P.nl2[(size_t)(g * G + hh) * P.q_pad + r] = -CUDART_INF_F;
@@ -262,15 +275,15 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
     if (!real)
         return; // the 8 lanes of a unit leave together
     const int row = P.q_begin + r;
-    if (g == 0 && sub == 0) {
+    if (g == 0 && sub == 0 && !P.rows_ready) {
         const int32_t mq = P.meta[row];
         P.mqp[r] = mq == META_NONE_K ? META_NONE_Q : mq;
     }
-    const int qt = r / BM, rr = r % BM;
-    const int ns = min(P.scount[qt], MAX_SINGLE);
     const __nv_bfloat16 *sq = sQ + (size_t)rl * row_elems, *sdo = sdO + (size_t)rl * row_elems,
                         *so = sO + (size_t)rl * row_elems;
     float *rnl2 = snl2 + rl * P.Hq, *rnd = snd + rl * P.Hq;
+    const int qt = r / BM, rr = r % BM;
+    const int ns = min(P.scount[qt], MAX_SINGLE);
     single_pass<true, KEYS>(P, 0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
     for (int i0 = KEYS; i0 < ns; i0 += KEYS) {
         __syncwarp(um); // lane 0's row values are visible to the unit's later passes
@@ -309,6 +322,7 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.scale = a.scale;
     P.scale_log2 = a.scale * 1.4426950408889634f;
     P.status = p.status;
+    P.rows_ready = a.rows_ready ? 1 : 0;
     // rows per block: up to 16 units of 8 lanes within 48 KB of shared memory (the headline shape,
     // 64 heads: one row, 25 KB, 64 threads; two rows per block measured the same)
     const size_t row_bytes = (size_t)a.Hq * (3 * 64 * 2 + 8);

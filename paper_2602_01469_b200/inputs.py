@@ -27,6 +27,9 @@ class Workload:
     seg_len: int | None = None   # fixed segment length in context tokens (overrides n_segments)
     seed: int = 0
     cod_r: float | None = None   # COD retention rate (Section 3): depth d keeps about n * r^d chains
+    # memory order inside a segment: "depth_major" = G0 | G1 | ... blocks (Figures 2-3);
+    # "anchor_major" = the depth-0 block, then the deeper tokens chain by chain (anchor, depth)
+    order: str = "depth_major"
 
     @property
     def total_tokens(self) -> int:
@@ -68,6 +71,9 @@ WORKLOADS = {
 # the paper's own example of Section 3.2: 8,192 tokens, K = 8, retention 0.8 (about 34K positions)
 WORKLOADS["gptoss_n8192_cod"] = Workload("gptoss_n8192_cod", (8192,), 8, 64, 8, 64, seed=60, cod_r=0.8)
 WORKLOADS["gptoss_n2048_profile"] = Workload("gptoss_n2048_profile", (2048,), 8, 64, 8, 64, seed=31)
+# the headline grid with a chain's tokens stored next to each other: a second workload, not the headline
+WORKLOADS["gptoss_n4096_anchor_major"] = Workload("gptoss_n4096_anchor_major", (4096,), 8, 64, 8, 64,
+                                                  seed=30, order="anchor_major")
 HEADLINE = "gptoss_n4096"
 
 
@@ -110,9 +116,14 @@ def segment_boundaries(n: int, n_segments: int = 1, seg_len: int | None = None) 
     return [(k * n) // n_segments for k in range(n_segments + 1)]
 
 
-def arrange_by_segment(anchor: np.ndarray, depth: np.ndarray, segment: np.ndarray):
-    """Memory order of one sequence: segments contiguous, depth-major inside a segment,
-    anchors ascending inside a depth.  Returns the permutation."""
+def arrange_by_segment(anchor: np.ndarray, depth: np.ndarray, segment: np.ndarray,
+                       order: str = "depth_major"):
+    """Memory order of one sequence: segments contiguous; inside a segment either depth-major
+    (anchors ascending inside a depth) or the depth-0 block followed by the deeper tokens
+    anchor-major, so that a chain's tokens are neighbours.  Returns the permutation."""
+    if order == "anchor_major":
+        return np.lexsort((depth, anchor, depth > 0, segment))
+    assert order == "depth_major"
     return np.lexsort((anchor, depth, segment))
 
 
@@ -182,7 +193,7 @@ def build_case(w: Workload, assign_fn):
             seg = np.asarray(assign_fn(a, d, w.K, bounds), dtype=np.int32)
         else:
             seg = np.zeros(a.shape[0], np.int32)
-        perm = arrange_by_segment(a, d, seg)
+        perm = arrange_by_segment(a, d, seg, w.order)
         a, d, seg = a[perm], d[perm], seg[perm]
         for p in partitions_from_layout(seg, d, offset=cu[-1]):
             p["seq"] = i

@@ -66,6 +66,9 @@ SMALL = [
     # COD-subsampled metadata (retention 0.7): ragged depth blocks, chain tiles that are no
     # diagonals, Algorithm 1 on nested position sets
     inputs.Workload("cod_segments", (700,), 6, 4, 2, 64, n_segments=2, seed=15, cod_r=0.7),
+    # a chain's tokens stored next to each other (depth-0 block, then anchor-major): the chain keys
+    # fall into the query tile's own neighbourhood instead of one-key-per-row tiles
+    inputs.Workload("anchor_major", (700,), 8, 4, 2, 64, n_segments=2, seed=17, order="anchor_major"),
     # more KV heads than the pair-by-pair kernels take: chain tiles stay on the tensor-core path
     inputs.Workload("many_kv_heads", (200,), 4, 24, 24, 64, seed=16),
 ]
@@ -199,7 +202,8 @@ def full_size_checks(case, n_rows=16, n_keys=6, seed=0):
             break
 
 
-@pytest.mark.parametrize("name", ["qwen3coder_n2048", "gptoss_n4096", "p90_n11008_s4"])
+@pytest.mark.parametrize("name", ["qwen3coder_n2048", "gptoss_n4096", "gptoss_n4096_anchor_major",
+                                  "p90_n11008_s4"])
 def test_partitioned_full_size(ctx, name):
     case = DeviceCase(inputs.WORKLOADS[name])
     run_partitioned(ctx, case)

@@ -48,6 +48,7 @@ SMALL = [
     inputs.Workload("cod_segments", (700,), 6, 4, 2, 64, n_segments=2, seed=15, cod_r=0.7),
     # more KV heads than the pair-by-pair kernels take: chain tiles stay on the tensor-core path
     inputs.Workload("many_kv_heads", (200,), 4, 24, 24, 64, seed=16),
+    inputs.Workload("anchor_major", (700,), 8, 4, 2, 64, n_segments=2, seed=17, order="anchor_major"),
 ]
 
 
