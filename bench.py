@@ -268,8 +268,25 @@ def run_cuda(args, w):
     bparts = [binding.Partition(p["seq"], p["q"], p["k"]) for p in parts]
     stream = torch.cuda.current_stream()
 
+    sharded = args.parallelism == "partitions"
+    if sharded:
+        # partition sharding: this rank's share of the query partitions against the full K / V,
+        # partial fp32 dK / dV sums completed by one all-reduce (NCCL), then rounded
+        from paper_2602_01469_b200 import sharding
+        my_parts = [bparts[i] for i in sharding.deal_partitions(parts, world)[rank]]
+        dK_acc = torch.zeros(T, w.n_kv_heads, w.head_dim, dtype=torch.float32, device=dev)
+        dV_acc = torch.zeros_like(dK_acc)
+
     def step():
-        binding.peagle_attn_partitioned(ctx, prob, bparts, Q, K, V, dO, O, LSE, dQ, dK, dV, stream)
+        if not sharded:
+            binding.peagle_attn_partitioned(ctx, prob, bparts, Q, K, V, dO, O, LSE, dQ, dK, dV, stream)
+            return
+        dK_acc.zero_()
+        dV_acc.zero_()
+        binding.peagle_attn_partitioned_acc(ctx, prob, my_parts, Q, K, V, dO, O, LSE, dQ, dK_acc,
+                                            dV_acc, stream)
+        sharding.sum_over_ranks([dK_acc, dV_acc], world)
+        binding.peagle_cast_grads(ctx, dK_acc, dV_acc, dK, dV, stream)
 
     def barrier():
         if world > 1:
@@ -301,7 +318,8 @@ def run_cuda(args, w):
     ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
     f_fwd, f_bwd = useful_flops(w)
-    value = replicas_value(world, f_fwd + f_bwd, ms_step)
+    # replicas: every rank does the whole workload; partitions: the ranks share one workload
+    value = replicas_value(1 if sharded else world, f_fwd + f_bwd, ms_step)
 
     # ---- end to end through the host entry point (pinned host buffers, copies timed)
     hQ, hK, hV, hdO = (t.pin_memory() for t in (Qc, Kc, Vc, dOc))
@@ -311,7 +329,16 @@ def run_cuda(args, w):
     hprob = binding.Problem(cu, anchor, depth, w.K, w.n_q_heads, w.n_kv_heads, w.head_dim, w.scale)
 
     def host_step():
-        binding.peagle_attn_partitioned_host(ctx, hprob, bparts, hQ, hK, hV, hdO, hO, hLSE, hdQ, hdK, hdV)
+        if not sharded:
+            binding.peagle_attn_partitioned_host(ctx, hprob, bparts, hQ, hK, hV, hdO, hO, hLSE, hdQ, hdK, hdV)
+            return
+        # sharded: host -> device copies, this rank's step, device -> host reads of its results
+        for d, h in ((Q, hQ), (K, hK), (V, hV), (dO, hdO)):
+            d.copy_(h, non_blocking=True)
+        step()
+        for h, d in ((hO, O), (hLSE, LSE), (hdQ, dQ), (hdK, dK), (hdV, dV)):
+            h.copy_(d, non_blocking=True)
+        torch.cuda.synchronize()
 
     host_step()
     barrier()
@@ -329,6 +356,11 @@ def run_cuda(args, w):
     if rank == 0:
         peaks, peak_kind = load_peaks()
         peak = float(peaks["bf16_tflops"])
+        if sharded:   # the timed launches are rank 0's: its partitions' share of the useful work
+            share = sum(int((anchor[b:e].astype(np.int64) + 1 + depth[b:e]).sum())
+                        for b, e in (parts[i]["q"] for i in sharding.deal_partitions(parts, world)[rank]))
+            share /= float(allowed_pairs(w))
+            f_fwd, f_bwd = f_fwd * share, f_bwd * share
         bwd_ms_launch = k_bwd_ms / max(n_bwd, 1)
         fwd_ms_launch = k_fwd_ms / max(n_fwd, 1)
         launches_per_step = max(n_bwd // args.steps, 1)
@@ -345,14 +377,15 @@ def run_cuda(args, w):
             "step_frac_of_peak": value / world / peak,
             "step_frac_of_sustained": value / world / float(peaks.get("bf16_tflops_sustained", peak)),
         }
+        f_fwd, f_bwd = useful_flops(w)
         cpu, _, _ = oracle_sample(w, args.cpu_seconds) if world == 1 and args.cpu_seconds > 0 else (None, 0, 0)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": config_dict(w, T, len(parts)),
+            "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": dict(config_dict(w, T, len(parts)), parallelism=args.parallelism),
             "clocks": clocks.summary(),
-            "e2e": {"value": world * (f_fwd + f_bwd) / e2e_s / 1e12, "unit": UNIT,
+            "e2e": {"value": (1 if sharded else world) * (f_fwd + f_bwd) / e2e_s / 1e12, "unit": UNIT,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": 1e3 * e2e_s},
             "gpu_launches": int(launches),
             "roofline": roofline,
@@ -424,6 +457,10 @@ def main():
     ap.add_argument("--workload", default=inputs.HEADLINE, choices=sorted(inputs.WORKLOADS))
     ap.add_argument("--op", default="attention", choices=["attention", "rope"],
                     help="attention: the hot path (default); rope: the rotary prologue side line")
+    ap.add_argument("--parallelism", default="replicas", choices=["replicas", "partitions"],
+                    help="with --gpus N > 1: N independent replicas of the workload (default), or one "
+                         "workload whose query partitions are dealt out over the ranks (dK / dV "
+                         "summed by an all-reduce); use a workload with several partitions")
     ap.add_argument("--cpu-seconds", type=float, default=15.0,
                     help="CPU time for the oracle baseline (0 = skip)")
     args = ap.parse_args()

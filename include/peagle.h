@@ -194,6 +194,24 @@ int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
                             void *dQ, void *dK, void *dV, void *stream);
 
 /*
+ * The driver's two halves for a caller that spreads the query partitions of a batch over several
+ * GPUs (Section 3.2: segments are independent given K and V; Section 5.1 trains on 8 GPUs).
+ * peagle_attn_partitioned_acc runs forward and backward of the given partitions like the driver
+ * but ADDS into the caller's fp32 accumulators dK_acc / dV_acc [T][n_kv_heads][head_dim] (dev,
+ * zeroed by the caller) and does not round them.  Each rank calls it with its share of the
+ * partitions and the full K / V, the accumulators are summed over the ranks (one collective over
+ * the whole arrays; keys that only one rank's queries see add zeros), and peagle_cast_grads rounds
+ * the sums to bf16: dK, dV [T][n_kv_heads][head_dim], count = T * n_kv_heads * head_dim (a
+ * multiple of 8).  O, LSE and dQ rows belong to the rank that owns their partition.
+ */
+int peagle_attn_partitioned_acc(peagle_ctx *ctx, const peagle_problem_t *prob,
+                                const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                                const void *K, const void *V, const void *dO, void *O, float *LSE,
+                                void *dQ, float *dK_acc, float *dV_acc, void *stream);
+int peagle_cast_grads(peagle_ctx *ctx, const float *dK_acc, const float *dV_acc, int64_t count,
+                      void *dK, void *dV, void *stream);
+
+/*
  * The same driver with HOST tensors (pinned memory, or the copies do not overlap anything).
  * K, V and the metadata go to the device first; then every partition's query range is cut into
  * slices of 2,048 rows that are themselves run as query partitions (Section 3.2's scheme: K / V

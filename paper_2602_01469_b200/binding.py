@@ -26,7 +26,7 @@ EXPORTS = [
     "peagle_attn_bwd", "peagle_attn_partitioned", "peagle_attn_partitioned_host",
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
     "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
-    "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd",
+    "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd", "peagle_attn_partitioned_acc", "peagle_cast_grads",
 ]
 
 
@@ -217,6 +217,21 @@ def peagle_attn_partitioned(ctx, prob: Problem, parts, Q, K, V, dO, O, LSE, dQ, 
     _check(lib().peagle_attn_partitioned(ctx.h, prob.ref(), arr, len(parts), _ptr(Q), _ptr(K),
                                          _ptr(V), _ptr(dO), _ptr(O), _ptr(LSE), _ptr(dQ), _ptr(dK),
                                          _ptr(dV), _stream(stream)), ctx.h)
+
+
+def peagle_attn_partitioned_acc(ctx, prob: Problem, parts, Q, K, V, dO, O, LSE, dQ, dK_acc, dV_acc,
+                                stream=None):
+    """Forward + backward of ``parts`` adding into the caller's fp32 dK / dV accumulators."""
+    arr = _partition_array(parts)
+    _check(lib().peagle_attn_partitioned_acc(ctx.h, prob.ref(), arr, len(parts), _ptr(Q), _ptr(K),
+                                             _ptr(V), _ptr(dO), _ptr(O), _ptr(LSE), _ptr(dQ),
+                                             _ptr(dK_acc), _ptr(dV_acc), _stream(stream)), ctx.h)
+
+
+def peagle_cast_grads(ctx, dK_acc, dV_acc, dK, dV, stream=None):
+    """Rounds fp32 dK / dV sums to bf16."""
+    _check(lib().peagle_cast_grads(ctx.h, _ptr(dK_acc), _ptr(dV_acc), ctypes.c_int64(dK_acc.numel()),
+                                   _ptr(dK), _ptr(dV), _stream(stream)), ctx.h)
 
 
 def peagle_attn_partitioned_host(ctx, prob: Problem, parts, Q, K, V, dO, O, LSE, dQ, dK, dV):

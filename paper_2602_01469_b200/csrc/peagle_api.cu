@@ -686,43 +686,15 @@ int peagle_attn_bwd(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_
     return run_bwd(ctx, prob, c, Q, K, V, O, dO, LSE, dQ, dK_acc, dV_acc, s);
 }
 
-int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
-                            const peagle_partition_t *parts, int32_t nparts, const void *Q,
-                            const void *K, const void *V, const void *dO, void *O, float *LSE,
-                            void *dQ, void *dK, void *dV, void *stream)
+// Runs forward + backward of the given partitions in order, adding into fp32 dK / dV accumulators.
+static int run_partitions(peagle_ctx *ctx, const peagle_problem_t *prob,
+                          const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                          const void *K, const void *V, const void *dO, void *O, float *LSE,
+                          void *dQ, float *dK_acc, float *dV_acc, cudaStream_t s)
 {
-    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV || (nparts > 0 && !parts))
-        return PEAGLE_ERR_NULL;
-    int rc = validate_problem(prob);
-    if (rc != PEAGLE_OK)
-        return rc;
-    if (nparts < 0)
-        return PEAGLE_ERR_BAD_RANGE;
-    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
-        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
-        return PEAGLE_ERR_ALIGN;
-    {   // check every partition before anything is launched
-        Call tmp;
-        for (int i = 0; i < nparts; ++i) {
-            rc = validate_partition(prob, &parts[i], tmp);
-            if (rc != PEAGLE_OK)
-                return rc;
-        }
-    }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    CK(cudaSetDevice(ctx->device));
-    const size_t n_kv = (size_t)prob->total_tokens * prob->n_kv_heads * prob->head_dim;
-    if (n_kv == 0)
-        return PEAGLE_OK;
-    rc = ensure(ctx, ctx->acc_buf, 2 * n_kv * sizeof(float), s);
-    if (rc != PEAGLE_OK)
-        return rc;
-    float *dK_acc = static_cast<float *>(ctx->acc_buf.ptr);
-    float *dV_acc = dK_acc + n_kv;
-    CK(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s));
     for (int i = 0; i < nparts; ++i) {
         Call c;
-        rc = plan_call(ctx, prob, &parts[i], true, s, c);
+        int rc = plan_call(ctx, prob, &parts[i], true, s, c);
         if (rc != PEAGLE_OK)
             return rc;
         // dO is known here, so the forward's epilogue leaves the backward's per-row values
@@ -740,7 +712,91 @@ int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
         if (rc != PEAGLE_OK)
             return rc;
     }
+    return PEAGLE_OK;
+}
+
+static int check_partitioned_args(const peagle_problem_t *prob, const peagle_partition_t *parts,
+                                  int32_t nparts)
+{
+    int rc = validate_problem(prob);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (nparts < 0)
+        return PEAGLE_ERR_BAD_RANGE;
+    Call tmp; // check every partition before anything is launched
+    for (int i = 0; i < nparts; ++i) {
+        rc = validate_partition(prob, &parts[i], tmp);
+        if (rc != PEAGLE_OK)
+            return rc;
+    }
+    return PEAGLE_OK;
+}
+
+int peagle_attn_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
+                            const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                            const void *K, const void *V, const void *dO, void *O, float *LSE,
+                            void *dQ, void *dK, void *dV, void *stream)
+{
+    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK || !dV || (nparts > 0 && !parts))
+        return PEAGLE_ERR_NULL;
+    int rc = check_partitioned_args(prob, parts, nparts);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK) || !aligned16(dV))
+        return PEAGLE_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CK(cudaSetDevice(ctx->device));
+    const size_t n_kv = (size_t)prob->total_tokens * prob->n_kv_heads * prob->head_dim;
+    if (n_kv == 0)
+        return PEAGLE_OK;
+    rc = ensure(ctx, ctx->acc_buf, 2 * n_kv * sizeof(float), s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    float *dK_acc = static_cast<float *>(ctx->acc_buf.ptr);
+    float *dV_acc = dK_acc + n_kv;
+    CK(cudaMemsetAsync(dK_acc, 0, 2 * n_kv * sizeof(float), s));
+    rc = run_partitions(ctx, prob, parts, nparts, Q, K, V, dO, O, LSE, dQ, dK_acc, dV_acc, s);
+    if (rc != PEAGLE_OK)
+        return rc;
     ctx->launches += launch_cast_grads(dK_acc, dV_acc, dK, dV, n_kv, s);
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int peagle_attn_partitioned_acc(peagle_ctx *ctx, const peagle_problem_t *prob,
+                                const peagle_partition_t *parts, int32_t nparts, const void *Q,
+                                const void *K, const void *V, const void *dO, void *O, float *LSE,
+                                void *dQ, float *dK_acc, float *dV_acc, void *stream)
+{
+    if (!ctx || !Q || !K || !V || !dO || !O || !LSE || !dQ || !dK_acc || !dV_acc ||
+        (nparts > 0 && !parts))
+        return PEAGLE_ERR_NULL;
+    int rc = check_partitioned_args(prob, parts, nparts);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) ||
+        !aligned16(dQ) || !aligned16(dK_acc) || !aligned16(dV_acc))
+        return PEAGLE_ERR_ALIGN;
+    CK(cudaSetDevice(ctx->device));
+    return run_partitions(ctx, prob, parts, nparts, Q, K, V, dO, O, LSE, dQ, dK_acc, dV_acc,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int peagle_cast_grads(peagle_ctx *ctx, const float *dK_acc, const float *dV_acc, int64_t count,
+                      void *dK, void *dV, void *stream)
+{
+    if (!ctx || !dK_acc || !dV_acc || !dK || !dV)
+        return PEAGLE_ERR_NULL;
+    if (count < 0 || count % 8 != 0)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (!aligned16(dK_acc) || !aligned16(dV_acc) || !aligned16(dK) || !aligned16(dV))
+        return PEAGLE_ERR_ALIGN;
+    if (count == 0)
+        return PEAGLE_OK;
+    CK(cudaSetDevice(ctx->device));
+    ctx->launches += launch_cast_grads(dK_acc, dV_acc, dK, dV, (size_t)count,
+                                       static_cast<cudaStream_t>(stream));
     CK(cudaGetLastError());
     return PEAGLE_OK;
 }

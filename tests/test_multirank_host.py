@@ -78,3 +78,73 @@ def test_kv_group_shards_partition_the_heads():
         assert (q_at, kv_at) == (hq, hkv)
     with pytest.raises(ValueError):
         kv_group_shard(6, 4, 0, 2)
+
+
+# ---------------------------------------------------------------- partition sharding
+def test_deal_partitions_covers_every_partition_once_and_balances():
+    from paper_2602_01469_b200 import inputs
+    from paper_2602_01469_b200.sharding import deal_partitions, partition_cost
+    from oracle import partition as opart
+    import numpy as np
+
+    def oracle_assign(anchor, depth, K, bounds):
+        P = inputs.position_sets(anchor, depth, K)
+        A, _, _ = opart.assign_segments(P, len(bounds) - 1, bounds[-1], B=bounds)
+        return np.array([A[d][a + d] for a, d in zip(anchor, depth)], np.int32)
+
+    _, _, _, parts = inputs.build_case(inputs.WORKLOADS["longtail_varlen"], oracle_assign)
+    assert len(parts) == 19
+    for world in (1, 2, 3, 8, 32):
+        mine = deal_partitions(parts, world)
+        assert sorted(i for m in mine for i in m) == list(range(len(parts)))
+        loads = [sum(partition_cost(parts[i]) for i in m) for m in mine]
+        if world <= 8:      # longest-first greedy: no rank exceeds the mean by more than one item
+            assert max(loads) <= sum(loads) / world + max(partition_cost(p) for p in parts)
+    with pytest.raises(ValueError):
+        deal_partitions(parts, 0)
+
+
+def _partition_worker(rank, world, port, out):
+    """Each rank runs the fp64 oracle on its share of the partitions; the partial dK / dV sums are
+    completed by the all-reduce the GPU path uses (gloo here)."""
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        import numpy as np
+        from oracle import partition as opart
+        from oracle import peagle_oracle as orc
+        from paper_2602_01469_b200 import inputs
+        from paper_2602_01469_b200.sharding import deal_partitions, sum_over_ranks
+
+        def oracle_assign(anchor, depth, K, bounds):
+            P = inputs.position_sets(anchor, depth, K)
+            A, _, _ = opart.assign_segments(P, len(bounds) - 1, bounds[-1], B=bounds)
+            return np.array([A[d][a + d] for a, d in zip(anchor, depth)], np.int32)
+
+        w = inputs.Workload("shard_parts", (41,), 4, 4, 2, 8, n_segments=3, seed=23)
+        cu, anchor, depth, parts = inputs.build_case(w, oracle_assign)
+        T = int(cu[-1])
+        Q, K, V, dO = inputs.make_tensors(T, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed, q_std=1.0)
+        dK = np.zeros((T, w.n_kv_heads, w.head_dim))
+        dV = np.zeros_like(dK)
+        dQ = np.zeros((T, w.n_q_heads, w.head_dim))
+        for i in deal_partitions(parts, world)[rank]:
+            rows = np.arange(*parts[i]["q"])
+            dQ[rows], _, _ = orc.attn_bwd(anchor, depth, Q, K, V, dO, 0.3, rows=rows,
+                                          kranges=parts[i]["k"], dK=dK, dV=dV)
+        tK, tV, tQ = torch.from_numpy(dK), torch.from_numpy(dV), torch.from_numpy(dQ)
+        sum_over_ranks([tK, tV, tQ], world)      # dQ rows are disjoint over ranks: the sum gathers them
+        want = orc.attn_bwd(anchor, depth, Q, K, V, dO, 0.3)
+        out[rank] = tuple(float(np.abs(a.numpy() - b).max()) for a, b in zip((tQ, tK, tV), want))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_two_ranks_partition_shards_sum_to_the_unpartitioned_gradients():
+    world, port = 2, _free_port()
+    with mp.Manager() as m:
+        out = m.dict()
+        mp.spawn(_partition_worker, args=(world, port, out), nprocs=world, join=True)
+        for rank in range(world):
+            assert max(out[rank]) < 1e-11, out[rank]
