@@ -254,6 +254,24 @@ int peagle_rope_qkv_bwd(peagle_ctx *ctx, const void *dQ, const void *dK, const v
                         void *d_qkv, void *stream);
 
 /*
+ * The projection products of the drafter layer (Section 2: a LLaMA-3-style layer; Section 3.2:
+ * every segment runs the layer on its tokens and on the depth-0 tokens before it).  bf16 operands,
+ * fp32 accumulation on the tensor cores:
+ *     C[m][n] (+)= sum_k A(m, k) * B(n, k),      m < M, n < N, k < K
+ * A(m, k) is A[m * lda + k], or A[k * lda + m] when a_transposed; B(n, k) is B[n * ldb + k], or
+ * B[k * ldb + n] when b_transposed.  With c_fp32_accumulate == 0, C is bf16 [M][ldc] and is
+ * written; otherwise C is fp32 [M][ldc] and the product is ADDED to it (launches on one stream are
+ * ordered; two calls that add into the same C from different streams race).  All dev, 16-byte
+ * aligned; lda, ldb, ldc (elements) and N multiples of 8; K >= 1.  Elements outside M x N are not
+ * touched.  So a linear layer Y = X W^T with W [d_out][d_in] is (A = X, B = W); its input gradient
+ * dX = dY W is (A = dY, B = W transposed, K = d_out); its weight gradient dW += dY^T X is
+ * (A = dY transposed, B = X transposed, K = rows, fp32 accumulate).  Asynchronous on `stream`.
+ */
+int peagle_gemm_bf16(peagle_ctx *ctx, const void *A, int64_t lda, int a_transposed, const void *B,
+                     int64_t ldb, int b_transposed, void *C, int64_t ldc, int c_fp32_accumulate,
+                     int32_t M, int32_t N, int32_t K, void *stream);
+
+/*
  * Algorithm 1, host only: segment of every token.  `boundaries` is host [S+1], context-token
  * positions with boundaries[0]=0 and boundaries[S]=n (Algorithm 1's B).  Depth 0 and 1 tokens
  * go by their position anchor+depth (a position at or beyond n stays in the last segment);

@@ -27,6 +27,7 @@ EXPORTS = [
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
     "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
     "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd", "peagle_attn_partitioned_acc", "peagle_cast_grads",
+    "peagle_gemm_bf16",
 ]
 
 
@@ -255,6 +256,13 @@ def peagle_rope_qkv_bwd(ctx, dQ, dK, dV, anchor, depth, Hq, Hkv, D, rope_base, d
     _check(lib().peagle_rope_qkv_bwd(ctx.h, _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(anchor), _ptr(depth),
                                      int(dQ.shape[0]), int(Hq), int(Hkv), int(D),
                                      ctypes.c_float(rope_base), _ptr(d_qkv), _stream(stream)), ctx.h)
+
+
+def peagle_gemm_bf16(ctx, A, lda, a_t, B, ldb, b_t, C, ldc, c_f32_add, M, N, K, stream=None):
+    """C[m][n] (+)= sum_k A(m,k) B(n,k); see include/peagle.h for the layouts."""
+    _check(lib().peagle_gemm_bf16(ctx.h, _ptr(A), ctypes.c_int64(lda), int(a_t), _ptr(B),
+                                  ctypes.c_int64(ldb), int(b_t), _ptr(C), ctypes.c_int64(ldc),
+                                  int(c_f32_add), int(M), int(N), int(K), _stream(stream)), ctx.h)
 
 
 def peagle_assign_segments(anchor, depth, K, boundaries):

@@ -801,6 +801,26 @@ int peagle_cast_grads(peagle_ctx *ctx, const float *dK_acc, const float *dV_acc,
     return PEAGLE_OK;
 }
 
+int peagle_gemm_bf16(peagle_ctx *ctx, const void *A, int64_t lda, int a_transposed, const void *B,
+                     int64_t ldb, int b_transposed, void *C, int64_t ldc, int c_fp32_accumulate,
+                     int32_t M, int32_t N, int32_t K, void *stream)
+{
+    if (!ctx || !A || !B || !C)
+        return PEAGLE_ERR_NULL;
+    if (M < 0 || N < 0 || K <= 0)
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (!aligned16(A) || !aligned16(B) || !aligned16(C))
+        return PEAGLE_ERR_ALIGN;
+    CK(cudaSetDevice(ctx->device));
+    const int n = launch_gemm(ctx->encode, A, lda, a_transposed, B, ldb, b_transposed, C, ldc,
+                              c_fp32_accumulate, M, N, K, ctx->status, static_cast<cudaStream_t>(stream));
+    if (n < 0)
+        return n;
+    ctx->launches += n;
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
 int peagle_attn_partitioned_host(peagle_ctx *ctx, const peagle_problem_t *prob,
                                  const peagle_partition_t *parts, int32_t nparts, const void *Q,
                                  const void *K, const void *V, const void *dO, void *O, float *LSE,

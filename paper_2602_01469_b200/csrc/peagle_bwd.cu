@@ -14,423 +14,22 @@
 //   dV  += P^T dO           P^T from tensor memory (bf16, over S^T), dO from shared memory (MN-major)
 //   dK  += dS^T Q           Q MN-major
 //   dQ   = dS K             dS^T read from shared memory as an MN-major A operand, K MN-major
-// Two kernels: bwd_kernel<D> (used for head_dim 128; every operand but P^T from shared memory,
-// one step at a time; warps 0-7 compute, warp 8 lane 0 issues the MMAs, warp 9 produces) and
-// bwd64_kernel (head_dim 64, below).
+// Two kernels with the same structure: bwd64_kernel (head_dim 64, below) and bwd128_kernel
+// (head_dim 128, peagle_bwd128.cu).
 #include <math_constants.h>
 
-#include "peagle_internal.h"
-#include "sm100_ptx.cuh"
+#include "peagle_bwd_common.cuh"
 
 namespace peagle {
 using namespace sm100;
 
 int make_bf16_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, int D, int H, int T);
-
-struct BwdParams {
-    const int2 *ktile;
-    const int4 *bitems;
-    const int *counters;
-    int *cursor; // device counter, zero at launch: next (work item, KV head) index to hand out
-    const int32_t *meta;
-    int *status;
-    int n_qt, q_begin, q_end, T;
-    const float *nl2, *nd; // [Hq][q_pad] -LSE*log2(e) and -Delta, padded rows (-inf, 0)
-    const int32_t *mqp;    // [q_pad] packed metadata of the partition's rows
-    int q_pad;             // n_qt * BM
-    float *dq_acc;         // [q_len][Hq][D]
-    float *dK_acc, *dV_acc;
-    int Hq, Hkv;
-    float scale, scale_log2;
-};
-
-template <int D>
-struct BwdCfg {
-    static constexpr int NSQ = (D == 64) ? 2 : 1;
-    static constexpr int PANELS = D / 64;
-    static constexpr int PANEL_BYTES = 128 * 128;
-    static constexpr int TILE_BYTES = PANELS * PANEL_BYTES;
-    static constexpr int OFF_K = 0;
-    static constexpr int OFF_V = TILE_BYTES;
-    static constexpr int OFF_DS = 2 * TILE_BYTES;                 // 2 panels: [key][q 0..63], [key][q 64..127]
-    static constexpr int OFF_Q = OFF_DS + 2 * PANEL_BYTES;        // ring of (Q, dO)
-    static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (lse2[128], delta[128], mq[128])
-    static constexpr int ROW_BYTES = 3 * 128 * 4;
-    static constexpr int OFF_BAR = OFF_ROW + NSQ * ROW_BYTES;
-    static constexpr int N_BAR = 2 * NSQ + 9;
-    static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;
-    static constexpr int SMEM_BYTES = OFF_MISC + 16 + 1024;
-    static constexpr int TM_S = 0;
-    static constexpr int TM_DP = 128;
-    static constexpr int TM_DQ = (D == 64) ? 256 : 128; // head_dim 128: dQ reuses the dP columns
-    static constexpr int TM_DK = (D == 64) ? 320 : 256;
-    static constexpr int TM_DV = (D == 64) ? 384 : 384;
-};
-
-__device__ __forceinline__ void red_add_v4(float *p, float a, float b, float c, float d)
-{
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(a), "f"(b), "f"(c),
-                 "f"(d)
-                 : "memory");
-}
-
-template <int D>
-__global__ void __launch_bounds__(320, 1)
-bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmdO,
-           const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
-           const BwdParams P)
-{
-    using C = BwdCfg<D>;
-    constexpr int NSQ = C::NSQ;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t sb = (raw + 1023u) & ~1023u;
-    uint8_t *sp = smem_raw + (sb - raw);
-    const uint32_t bar0 = sb + C::OFF_BAR;
-    auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
-    constexpr int B_QFULL = 0, B_QEMPTY = NSQ, B_KVFULL = 2 * NSQ, B_KVEMPTY = B_KVFULL + 1,
-                  B_ACCFREE = B_KVFULL + 2, B_SFULL = B_KVFULL + 3, B_DPFULL = B_KVFULL + 4,
-                  B_PFULL = B_KVFULL + 5, B_DSFULL = B_KVFULL + 6, B_DQFULL = B_KVFULL + 7,
-                  B_DQEMPTY = B_KVFULL + 8;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_MISC);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_MISC + 4);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = P.Hq / P.Hkv;
-    const int total_items = P.counters[1] * P.Hkv;
-
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int s = 0; s < NSQ; ++s) {
-            mbar_init(BAR(B_QFULL + s), 1);
-            mbar_init(BAR(B_QEMPTY + s), 1);
-        }
-        mbar_init(BAR(B_KVFULL), 1);
-        mbar_init(BAR(B_KVEMPTY), 1);
-        mbar_init(BAR(B_ACCFREE), 256);
-        mbar_init(BAR(B_SFULL), 1);
-        mbar_init(BAR(B_DPFULL), 1);
-        mbar_init(BAR(B_PFULL), 256);
-        mbar_init(BAR(B_DSFULL), 256);
-        mbar_init(BAR(B_DQFULL), 1);
-        mbar_init(BAR(B_DQEMPTY), 256);
-        fence_mbar_init();
-    }
-    if (warp == 8) {
-        tmem_alloc(sb + C::OFF_MISC, 512);
-        tmem_relinquish();
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *tmem_slot;
-
-    if (warp == 9) {
-        // ------------------------------------------------------------ producer
-        if (lane == 0) {
-            tma_prefetch_desc(&tmQ);
-            tma_prefetch_desc(&tmdO);
-            tma_prefetch_desc(&tmK);
-            tma_prefetch_desc(&tmV);
-        }
-        int it = 0, w = 0;
-        bool ok = true;
-        for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
-            const int4 item = P.bitems[idx / P.Hkv];
-            const int g = idx % P.Hkv;
-            const int kt = item.x;
-            const int2 ktile = P.ktile[kt];
-            if (lane == 0) {
-                ok = mbar_wait(BAR(B_KVEMPTY), (w & 1) ^ 1, abort_flag);
-                if (ok) {
-                    mbar_arrive_expect_tx(BAR(B_KVFULL), 2 * C::TILE_BYTES);
-                    for (int pn = 0; pn < C::PANELS; ++pn) {
-                        tma_load_3d(sb + C::OFF_K + pn * C::PANEL_BYTES, &tmK, BAR(B_KVFULL), pn * 64,
-                                    g, ktile.x);
-                        tma_load_3d(sb + C::OFF_V + pn * C::PANEL_BYTES, &tmV, BAR(B_KVFULL), pn * 64,
-                                    g, ktile.x);
-                    }
-                }
-            }
-            ok = __all_sync(0xffffffffu, ok);
-            for (unsigned em = (unsigned)item.z & 0xffu; ok && em; em &= em - 1) {
-                const int qt = item.y * BWD_CQ + (__ffs(em) - 1);
-                const int row0 = P.q_begin + qt * BM;
-                for (int hh = 0; ok && hh < G; ++hh, ++it) {
-                    const int h = g * G + hh;
-                    const int st = it % NSQ, ph = (it / NSQ) & 1;
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QEMPTY + st), ph ^ 1, abort_flag));
-                    if (!ok)
-                        break;
-                    float *rowbuf = reinterpret_cast<float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
-                    for (int i = lane; i < BM; i += 32) {
-                        const int row = row0 + i;
-                        const size_t ri = (size_t)h * P.q_pad + (row - P.q_begin);
-                        rowbuf[i] = -P.nl2[ri];
-                        rowbuf[128 + i] = -P.nd[ri];
-                        reinterpret_cast<int *>(rowbuf)[256 + i] = P.mqp[row - P.q_begin];
-                    }
-                    __syncwarp();
-                    if (lane == 0) {
-                        mbar_arrive_expect_tx(BAR(B_QFULL + st), 2 * C::TILE_BYTES);
-                        const uint32_t qa = sb + C::OFF_Q + st * 2 * C::TILE_BYTES;
-                        for (int pn = 0; pn < C::PANELS; ++pn) {
-                            tma_load_3d(qa + pn * C::PANEL_BYTES, &tmQ, BAR(B_QFULL + st), pn * 64, h,
-                                        row0);
-                            tma_load_3d(qa + C::TILE_BYTES + pn * C::PANEL_BYTES, &tmdO,
-                                        BAR(B_QFULL + st), pn * 64, h, row0);
-                        }
-                    }
-                }
-            }
-        }
-    } else if (warp == 8) {
-        // ------------------------------------------------------------ MMA issue
-        if (lane == 0) {
-            constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
-            constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
-            constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
-            const uint32_t ka = sb + C::OFF_K, va = sb + C::OFF_V, dsa = sb + C::OFF_DS;
-            int it = 0, w = 0;
-            bool ok = true;
-            for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
-                const int4 item = P.bitems[idx / P.Hkv];
-                const int n_it = item.w * G;
-                ok = mbar_wait(BAR(B_KVFULL), w & 1, abort_flag) &&
-                     mbar_wait(BAR(B_ACCFREE), (w & 1) ^ 1, abort_flag);
-                for (int i = 0; ok && i < n_it; ++i, ++it) {
-                    const int st = it % NSQ, ph = (it / NSQ) & 1;
-                    const uint32_t qa = sb + C::OFF_Q + st * 2 * C::TILE_BYTES;
-                    const uint32_t doa = qa + C::TILE_BYTES;
-                    ok = mbar_wait(BAR(B_QFULL + st), ph, abort_flag);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
-                        mma_ss(tmem + C::TM_S, smem_desc_sw128(ka + off, 16, 1024),
-                               smem_desc_sw128(qa + off, 16, 1024), IDESC_S, k > 0);
-                    }
-                    tc_commit(BAR(B_SFULL));
-                    if (D == 128) { // dQ of the previous iteration lives in the dP columns
-                        ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, abort_flag);
-                        if (!ok)
-                            break;
-                        tc_fence_after();
-                    }
-#pragma unroll
-                    for (int k = 0; k < D / 16; ++k) {
-                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
-                        mma_ss(tmem + C::TM_DP, smem_desc_sw128(va + off, 16, 1024),
-                               smem_desc_sw128(doa + off, 16, 1024), IDESC_S, k > 0);
-                    }
-                    tc_commit(BAR(B_DPFULL));
-                    ok = mbar_wait(BAR(B_PFULL), it & 1, abort_flag);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        mma_ts(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
-                               smem_desc_sw128(doa + k * 2048, C::PANEL_BYTES, 1024), IDESC_KV,
-                               i > 0 || k > 0);
-                    ok = mbar_wait(BAR(B_DSFULL), it & 1, abort_flag);
-                    if (ok && D == 64)
-                        ok = mbar_wait(BAR(B_DQEMPTY), (it & 1) ^ 1, abort_flag);
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        const uint32_t off = (k / 4) * C::PANEL_BYTES + (k % 4) * 32;
-                        mma_ss(tmem + C::TM_DK, smem_desc_sw128(dsa + off, 16, 1024),
-                               smem_desc_sw128(qa + k * 2048, C::PANEL_BYTES, 1024), IDESC_KV,
-                               i > 0 || k > 0);
-                    }
-#pragma unroll
-                    for (int k = 0; k < 8; ++k)
-                        mma_ss(tmem + C::TM_DQ, smem_desc_sw128(dsa + k * 2048, C::PANEL_BYTES, 1024),
-                               smem_desc_sw128(ka + k * 2048, C::PANEL_BYTES, 1024), IDESC_DQ, k > 0);
-                    tc_commit(BAR(B_DQFULL));
-                    tc_commit(BAR(B_QEMPTY + st));
-                }
-                if (ok)
-                    tc_commit(BAR(B_KVEMPTY));
-            }
-        }
-    } else {
-        // ------------------------------------------------------------ compute (warps 0-7)
-        const int wg = warp >> 2;
-        const int r = threadIdx.x & 127; // key lane for S/dP/dK/dV, query row for dQ
-        const uint32_t lane_sel = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t tS = tmem + lane_sel + C::TM_S + wg * 64;
-        const uint32_t tDP = tmem + lane_sel + C::TM_DP + wg * 64;
-        const uint32_t tDQ = tmem + lane_sel + C::TM_DQ + wg * (D / 2);
-        const uint32_t tACC = tmem + lane_sel + (wg == 0 ? C::TM_DK : C::TM_DV);
-        const size_t q_len = (size_t)(P.q_end - P.q_begin);
-        int it = 0, w = 0;
-        bool ok = true;
-        for (int idx = blockIdx.x; ok && idx < total_items; idx += gridDim.x, ++w) {
-            const int4 item = P.bitems[idx / P.Hkv];
-            const int g = idx % P.Hkv;
-            const int kt = item.x;
-            const int2 ktile = P.ktile[kt];
-            const int32_t mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
-            for (unsigned em = (unsigned)item.z & 0xffu; ok && em; em &= em - 1) {
-                const int eb = __ffs(em) - 1;
-                const int row0 = P.q_begin + (item.y * BWD_CQ + eb) * BM;
-                const bool full = ((unsigned)item.z >> (8 + eb)) & 1u;
-                for (int hh = 0; ok && hh < G; ++hh, ++it) {
-                    const int h = g * G + hh;
-                    const int st = it % NSQ, ph = (it / NSQ) & 1;
-                    const float *rowbuf =
-                        reinterpret_cast<const float *>(sp + C::OFF_ROW + st * C::ROW_BYTES);
-                    const float4 *lse4 = reinterpret_cast<const float4 *>(rowbuf + wg * 64);
-                    const float4 *dl4 = reinterpret_cast<const float4 *>(rowbuf + 128 + wg * 64);
-                    const int4 *mq4 = reinterpret_cast<const int4 *>(rowbuf + 256 + wg * 64);
-                    // ---- P^T
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL), it & 1, abort_flag) &&
-                                                     mbar_wait(BAR(B_QFULL + st), ph, abort_flag));
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    uint32_t sr[2][32];
-                    tmem_ld32(tS, sr[0]);
-                    tmem_ld32(tS + 32, sr[1]);
-                    tmem_wait_ld();
-                    float p[64];
-#pragma unroll
-                    for (int c = 0; c < 64; c += 4) {
-                        const float4 l = lse4[c >> 2];
-                        p[c + 0] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 0) & 31]), P.scale_log2, -l.x));
-                        p[c + 1] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 1) & 31]), P.scale_log2, -l.y));
-                        p[c + 2] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 2) & 31]), P.scale_log2, -l.z));
-                        p[c + 3] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 3) & 31]), P.scale_log2, -l.w));
-                    }
-                    if (!full) {
-#pragma unroll
-                        for (int c = 0; c < 64; c += 4) {
-                            const int4 mq = mq4[c >> 2];
-                            if (!allowed_packed(mq.x, mk)) p[c + 0] = 0.f;
-                            if (!allowed_packed(mq.y, mk)) p[c + 1] = 0.f;
-                            if (!allowed_packed(mq.z, mk)) p[c + 2] = 0.f;
-                            if (!allowed_packed(mq.w, mk)) p[c + 3] = 0.f;
-                        }
-                    }
-                    {
-                        uint32_t pk[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            pk[i] = pack_bf16x2(p[2 * i], p[2 * i + 1]);
-                        tmem_st32(tS, pk); // packed P^T over the first half of this group's S^T columns
-                    }
-                    tmem_wait_st();
-                    tc_fence_before();
-                    mbar_arrive(BAR(B_PFULL));
-                    // ---- dS^T
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DPFULL), it & 1, abort_flag));
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    tmem_ld32(tDP, sr[0]);
-                    tmem_ld32(tDP + 32, sr[1]);
-                    tmem_wait_ld();
-                    {
-                        uint8_t *dsrow = sp + C::OFF_DS + wg * C::PANEL_BYTES + r * 128;
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) { // 16-byte chunk j = query columns 8j .. 8j+7
-                            const float4 d0 = dl4[2 * j], d1 = dl4[2 * j + 1];
-                            const int c = 8 * j;
-                            uint4 v;
-                            v.x = pack_bf16x2(p[c + 0] * (__uint_as_float(sr[c >> 5][(c + 0) & 31]) - d0.x),
-                                              p[c + 1] * (__uint_as_float(sr[c >> 5][(c + 1) & 31]) - d0.y));
-                            v.y = pack_bf16x2(p[c + 2] * (__uint_as_float(sr[c >> 5][(c + 2) & 31]) - d0.z),
-                                              p[c + 3] * (__uint_as_float(sr[c >> 5][(c + 3) & 31]) - d0.w));
-                            v.z = pack_bf16x2(p[c + 4] * (__uint_as_float(sr[c >> 5][(c + 4) & 31]) - d1.x),
-                                              p[c + 5] * (__uint_as_float(sr[c >> 5][(c + 5) & 31]) - d1.y));
-                            v.w = pack_bf16x2(p[c + 6] * (__uint_as_float(sr[c >> 5][(c + 6) & 31]) - d1.z),
-                                              p[c + 7] * (__uint_as_float(sr[c >> 5][(c + 7) & 31]) - d1.w));
-                            *reinterpret_cast<uint4 *>(dsrow + ((j ^ (r & 7)) << 4)) = v;
-                        }
-                    }
-                    fence_proxy_async_smem();
-                    tc_fence_before();
-                    mbar_arrive(BAR(B_DSFULL));
-                    // ---- dQ of this (query tile, head): add to the fp32 staging buffer
-                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DQFULL), it & 1, abort_flag));
-                    if (!ok)
-                        break;
-                    tc_fence_after();
-                    {
-                        const int row = row0 + r;
-                        float *dst = P.dq_acc + ((size_t)(row - P.q_begin) * P.Hq + h) * D + wg * (D / 2);
-#pragma unroll
-                        for (int c = 0; c < D / 64; ++c) {
-                            uint32_t o[32];
-                            tmem_ld32(tDQ + c * 32, o);
-                            tmem_wait_ld();
-                            if (row < P.q_end) {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 4)
-                                    red_add_v4(dst + c * 32 + i, __uint_as_float(o[i]) * P.scale,
-                                               __uint_as_float(o[i + 1]) * P.scale,
-                                               __uint_as_float(o[i + 2]) * P.scale,
-                                               __uint_as_float(o[i + 3]) * P.scale);
-                            }
-                        }
-                    }
-                    tc_fence_before();
-                    mbar_arrive(BAR(B_DQEMPTY));
-                }
-            }
-            if (!ok)
-                break;
-            // ---- end of item: dK (group 0) / dV (group 1) of this key tile
-            {
-                float *acc = (wg == 0 ? P.dK_acc : P.dV_acc) +
-                             ((size_t)(ktile.x + r) * P.Hkv + g) * D;
-                const float f = (wg == 0) ? P.scale : 1.f;
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint32_t o[32];
-                    tmem_ld32(tACC + c * 32, o);
-                    tmem_wait_ld();
-                    if (r < ktile.y) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            red_add_v4(acc + c * 32 + i, __uint_as_float(o[i]) * f,
-                                       __uint_as_float(o[i + 1]) * f, __uint_as_float(o[i + 2]) * f,
-                                       __uint_as_float(o[i + 3]) * f);
-                    }
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(BAR(B_ACCFREE));
-        }
-        (void)q_len;
-    }
-
-    // ------------------------------------------------------------ teardown
-    tc_fence_before();
-    __syncthreads();
-    if (*abort_flag) {
-        if (threadIdx.x == 0)
-            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
-        const uint64_t t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) {
-        }
-        __syncthreads();
-    }
-    if (warp == 8) {
-        __syncwarp();
-        tc_fence_after();
-        tmem_dealloc(tmem, 512);
-    }
-}
+int launch_bwd128_main(const CUtensorMap &tmQ, const CUtensorMap &tmdO, const CUtensorMap &tmK,
+                       const CUtensorMap &tmV, const CUtensorMap &tmDQ, const BwdParams &P, int n_sm,
+                       cudaStream_t s);
 
 // ---------------------------------------------------------------------------------------------
-// head_dim 64: software-pipelined variant.  The MMA warp runs one step ahead of the compute warps
+// head_dim 64.  The MMA warp runs one step ahead of the compute warps
 // inside a work item:
 //   while the compute warps turn S^T(i) into P^T(i):   dK(i-1), dQ(i-1), dP^T(i)
 //   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
@@ -460,86 +59,6 @@ struct Bwd64Cfg {
     // first half of each group's S^T columns and dS^T (bf16) the first half of its dP^T columns.
     static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_K = 320, TM_V = 352, TM_DK = 384,
                          TM_DV = 448;
-};
-
-// Walks the (work item, query tile, head) iterations of one CTA in execution order.  Work items
-// are handed out dynamically: the producer warp takes the next (item, KV head) index from a global
-// cursor and publishes it in a four-slot queue in shared memory; the other roles read it there.
-// A CTA that falls behind therefore takes fewer items, and the CTAs running at any time work on a
-// contiguous window of the chunk-major item list (their shared Q / dO rows and dQ staging rows
-// stay in L2), instead of drifting apart as with a static round-robin.
-struct BwdWalk {
-    const int4 *bitems;
-    int *cursor;
-    volatile int *wq;
-    volatile int *abort;
-    uint32_t wqbar;
-    int idx, total, Hkv, G, lane;
-    bool fetcher;
-    int kt, g, c, w;
-    unsigned mask, em;
-    int hh;
-    bool valid;
-    __device__ void load()
-    {
-        const int slot = w & 3;
-        if (fetcher) { // the whole producer warp, convergent
-            int v = 0;
-            if (lane == 0)
-                v = atomicAdd(cursor, 1);
-            v = __shfl_sync(0xffffffffu, v, 0);
-            idx = v < total ? v : -1;
-            if (lane == 0) {
-                wq[slot] = idx;
-                sm100::mbar_arrive(wqbar + 8u * slot);
-            }
-        } else {
-            // slot w & 3 was last used four items ago; no role is more than two items behind
-            idx = sm100::mbar_wait(wqbar + 8u * slot, (w >> 2) & 1, abort) ? wq[slot] : -1;
-        }
-        valid = idx >= 0;
-        if (!valid)
-            return;
-        const int4 item = bitems[idx / Hkv];
-        g = idx % Hkv;
-        kt = item.x;
-        c = item.y;
-        mask = (unsigned)item.z;
-        em = mask & 0xffu;
-        hh = 0;
-    }
-    __device__ void init(const BwdParams &P, volatile int *queue, uint32_t queue_bar,
-                         volatile int *abort_flag, bool is_fetcher, int lane_id)
-    {
-        bitems = P.bitems;
-        cursor = P.cursor;
-        wq = queue;
-        wqbar = queue_bar;
-        abort = abort_flag;
-        fetcher = is_fetcher;
-        lane = lane_id;
-        Hkv = P.Hkv;
-        G = P.Hq / P.Hkv;
-        total = P.counters[1] * P.Hkv;
-        w = 0;
-        load();
-    }
-    __device__ bool first() const { return hh == 0 && em == (mask & 0xffu); }
-    __device__ bool last() const { return hh == G - 1 && (em & (em - 1)) == 0; }
-    __device__ int qt() const { return c * BWD_CQ + (__ffs(em) - 1); }
-    __device__ bool full() const { return (mask >> (8 + __ffs(em) - 1)) & 1u; }
-    __device__ int head() const { return g * G + hh; }
-    __device__ void next()
-    {
-        if (++hh == G) {
-            hh = 0;
-            em &= em - 1;
-            if (em == 0) {
-                ++w;
-                load();
-            }
-        }
-    }
 };
 
 __global__ void __launch_bounds__(512, 1)
@@ -1177,21 +696,16 @@ static int launch_bwd_t(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int 
         P.Hkv = a.Hkv;
         P.scale = a.scale;
         P.scale_log2 = a.scale * 1.4426950408889634f;
-        {   // per device, so set before every launch (host time only)
-            const cudaError_t e =
-                (D == 64) ? cudaFuncSetAttribute(bwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 Bwd64Cfg::SMEM_BYTES)
-                          : cudaFuncSetAttribute(bwd_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 BwdCfg<D>::SMEM_BYTES);
-            if (e != cudaSuccess)
-                return PEAGLE_ERR_CUDA;
-        }
+        // per device, so set before every launch (host time only)
+        if (D == 64 && cudaFuncSetAttribute(bwd64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            Bwd64Cfg::SMEM_BYTES) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
         if (ev0)
             cudaEventRecord(ev0, s);
         if (D == 64)
             bwd64_kernel<<<n_sm, 512, Bwd64Cfg::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, tmDQ, P);
-        else
-            bwd_kernel<D><<<n_sm, 320, BwdCfg<D>::SMEM_BYTES, s>>>(tmQ, tmdO, tmK, tmV, P);
+        else if (launch_bwd128_main(tmQ, tmdO, tmK, tmV, tmDQ, P, n_sm, s) < 0)
+            return PEAGLE_ERR_CUDA;
         if (ev1)
             cudaEventRecord(ev1, s);
         ++launches;

@@ -1,0 +1,242 @@
+// Dense bf16 projection products of the drafter layer on sm_100a (Section 2: a LLaMA-3-style layer;
+// Section 3.2: every segment runs the layer on its own tokens and on the depth-0 tokens before
+// it, so the K / V projections of those tokens are recomputed per segment).
+//
+//   C[m][n] (+)= sum_k A(m, k) * B(n, k),   bf16 operands, fp32 accumulation in tensor memory
+//
+// Each operand is either stored with k contiguous ("K-major": A[m][k], B[n][k]) or transposed
+// ("MN-major": A[k][m], B[k][n]); the three products of a linear layer are
+//   forward      Y  = X W^T      A = X  [rows][d_in]  K-major,  B = W [d_out][d_in] K-major
+//   input grad   dX = dY W       A = dY [rows][d_out] K-major,  B = W [d_out][d_in] MN-major (k = d_out)
+//   weight grad  dW = dY^T X     A = dY [rows][d_out] MN-major, B = X [rows][d_in]  MN-major (k = rows)
+// One CTA computes one 128 x 128 tile of C: warp 0 loads 64-wide k slabs of A and B by TMA into a
+// ring of stages (128-byte swizzle), warp 1 lane 0 issues tcgen05.mma (four k = 16 products per
+// slab) and releases the stages by commits, warps 2-5 read the accumulator when the last commit
+// arrives and either store bf16 rows or add into an fp32 C (tiles of one launch are disjoint and
+// launches on a stream are ordered, so the addition is a plain load-add-store).
+#include "peagle_internal.h"
+#include "sm100_ptx.cuh"
+
+namespace peagle {
+using namespace sm100;
+
+namespace {
+
+constexpr int GT = 128;      // tile of C
+constexpr int GK = 64;       // k slab
+constexpr int G_STAGES = 4;
+constexpr int G_TILE_BYTES = GT * GK * 2; // 16 KB per operand and stage
+constexpr int G_OFF_BAR = 2 * G_STAGES * G_TILE_BYTES;
+constexpr int G_SMEM = G_OFF_BAR + (2 * G_STAGES + 1) * 8 + 32 + 1024;
+
+struct GemmParams {
+    int M, N, K;
+    int a_t, b_t;  // 1: operand stored transposed (MN-major)
+    int c_f32_add; // 0: C bf16, stored; 1: C fp32, added to
+    void *C;
+    long long ldc;
+    int *status;
+};
+
+__global__ void __launch_bounds__(192, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+            const GemmParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u;
+    uint8_t *sp = smem_raw + (sb - raw);
+    const uint32_t bar0 = sb + G_OFF_BAR;
+    auto FULL = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto EMPTY = [&](int s) { return bar0 + 8u * (uint32_t)(G_STAGES + s); };
+    const uint32_t ACC = bar0 + 8u * (2 * G_STAGES);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + G_OFF_BAR + (2 * G_STAGES + 1) * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + G_OFF_BAR + (2 * G_STAGES + 1) * 8 + 4);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.y * GT, n0 = blockIdx.x * GT;
+    const int n_k = (P.K + GK - 1) / GK;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < G_STAGES; ++s) {
+            mbar_init(FULL(s), 1);
+            mbar_init(EMPTY(s), 1);
+        }
+        mbar_init(ACC, 1);
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), 128);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer
+        if (lane == 0) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            for (int i = 0; i < n_k; ++i) {
+                const int s = i % G_STAGES;
+                if (!mbar_wait(EMPTY(s), ((i / G_STAGES) & 1) ^ 1, abort_flag))
+                    break;
+                mbar_arrive_expect_tx(FULL(s), 2 * G_TILE_BYTES);
+                const uint32_t a = sb + s * 2 * G_TILE_BYTES, b = a + G_TILE_BYTES;
+                const int k0 = i * GK;
+                if (!P.a_t) {
+                    tma_load_2d(a, &tmA, FULL(s), k0, m0); // [128 m][64 k]
+                } else {                                    // two panels [64 k][64 m]
+                    tma_load_2d(a, &tmA, FULL(s), m0, k0);
+                    tma_load_2d(a + G_TILE_BYTES / 2, &tmA, FULL(s), m0 + 64, k0);
+                }
+                if (!P.b_t) {
+                    tma_load_2d(b, &tmB, FULL(s), k0, n0);
+                } else {
+                    tma_load_2d(b, &tmB, FULL(s), n0, k0);
+                    tma_load_2d(b + G_TILE_BYTES / 2, &tmB, FULL(s), n0 + 64, k0);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------ MMA issue
+        if (lane == 0) {
+            const uint32_t idesc = idesc_bf16_f32(GT, GT, P.a_t, P.b_t);
+            // K-major: a k = 16 slice is 32 bytes further inside the 128-byte rows; MN-major: 16
+            // rows (2,048 bytes) further, the second 64-wide panel half a tile on
+            const uint32_t a_step = P.a_t ? 128u : 2u, b_step = P.b_t ? 128u : 2u;
+            bool ok = true;
+            for (int i = 0; ok && i < n_k; ++i) {
+                const int s = i % G_STAGES;
+                ok = mbar_wait(FULL(s), (i / G_STAGES) & 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                const uint32_t a = sb + s * 2 * G_TILE_BYTES, b = a + G_TILE_BYTES;
+                const uint32_t a_lo = desc_lo_sw128(a, P.a_t ? G_TILE_BYTES / 2 : 16);
+                const uint32_t b_lo = desc_lo_sw128(b, P.b_t ? G_TILE_BYTES / 2 : 16);
+#pragma unroll
+                for (int k = 0; k < GK / 16; ++k)
+                    mma_ss_lo(tmem, a_lo + k * a_step, b_lo + k * b_step, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                tc_commit(EMPTY(s));
+            }
+            if (ok)
+                tc_commit(ACC);
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2-5)
+        const int q = warp & 3; // tensor-memory lane quarter this warp may read
+        const int m = m0 + q * 32 + lane;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(ACC, 0, abort_flag));
+        if (ok) {
+            tc_fence_after();
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+#pragma unroll 1
+            for (int c = 0; c < GT / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(trow + c * 32, o);
+                tmem_wait_ld();
+                const int n = n0 + c * 32;
+                if (m >= P.M)
+                    continue;
+                if (!P.c_f32_add) {
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(P.C) + (size_t)m * P.ldc + n;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        if (n + i < P.N) { // N is a multiple of 8
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(o[i + 0]), __uint_as_float(o[i + 1]));
+                            v.y = pack_bf16x2(__uint_as_float(o[i + 2]), __uint_as_float(o[i + 3]));
+                            v.z = pack_bf16x2(__uint_as_float(o[i + 4]), __uint_as_float(o[i + 5]));
+                            v.w = pack_bf16x2(__uint_as_float(o[i + 6]), __uint_as_float(o[i + 7]));
+                            *reinterpret_cast<uint4 *>(dst + i) = v;
+                        }
+                    }
+                } else {
+                    float *dst = static_cast<float *>(P.C) + (size_t)m * P.ldc + n;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        if (n + i < P.N) {
+                            float4 v = *reinterpret_cast<float4 *>(dst + i);
+                            v.x += __uint_as_float(o[i + 0]);
+                            v.y += __uint_as_float(o[i + 1]);
+                            v.z += __uint_as_float(o[i + 2]);
+                            v.w += __uint_as_float(o[i + 3]);
+                            *reinterpret_cast<float4 *>(dst + i) = v;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------ teardown
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
+        const uint64_t t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) {
+        }
+        __syncthreads();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem, 128);
+    }
+}
+
+// Tensor map of a row-major bf16 matrix [rows][cols] with leading dimension ld (elements).
+int matrix_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, long long rows, long long cols,
+               long long ld, int box_cols, int box_rows)
+{
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box,
+               estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS
+               ? 0
+               : -1;
+}
+
+} // namespace
+
+// Returns the number of kernels launched (1), 0 for an empty product, or a negative status.
+int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const void *B, long long ldb,
+                int b_t, void *C, long long ldc, int c_f32_add, int M, int N, int K, int *status,
+                cudaStream_t s)
+{
+    if (M <= 0 || N <= 0)
+        return 0;
+    if (K <= 0 || (N % 8) || (lda % 8) || (ldb % 8) || (ldc % (c_f32_add ? 4 : 8)))
+        return PEAGLE_ERR_BAD_SHAPE;
+    CUtensorMap tmA, tmB;
+    // K-major operand [R][K]: boxes of 64 k x 128 rows; transposed [K][R]: boxes of 64 r x 64 k
+    const int ra = a_t ? matrix_map(enc, &tmA, A, K, M, lda, 64, 64) : matrix_map(enc, &tmA, A, M, K, lda, 64, GT);
+    const int rb = b_t ? matrix_map(enc, &tmB, B, K, N, ldb, 64, 64) : matrix_map(enc, &tmB, B, N, K, ldb, 64, GT);
+    if (ra || rb)
+        return PEAGLE_ERR_CUDA;
+    GemmParams P;
+    P.M = M;
+    P.N = N;
+    P.K = K;
+    P.a_t = a_t ? 1 : 0;
+    P.b_t = b_t ? 1 : 0;
+    P.c_f32_add = c_f32_add ? 1 : 0;
+    P.C = C;
+    P.ldc = ldc;
+    P.status = status;
+    if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM) != cudaSuccess)
+        return PEAGLE_ERR_CUDA;
+    dim3 grid((unsigned)((N + GT - 1) / GT), (unsigned)((M + GT - 1) / GT));
+    gemm_kernel<<<grid, 192, G_SMEM, s>>>(tmA, tmB, P);
+    return 1;
+}
+
+} // namespace peagle

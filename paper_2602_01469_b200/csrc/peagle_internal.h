@@ -116,6 +116,13 @@ int launch_rope(bool backward, const void *fused_in, void *fused_out, const void
                 const int32_t *anchor, const int32_t *depth, int T, int Hq, int Hkv, int D,
                 float base, int n_sm, cudaStream_t s);
 
+// C[m][n] (+)= sum_k A(m,k) B(n,k) in bf16 with fp32 accumulation (peagle_gemm.cu).  a_t / b_t: the
+// operand is stored transposed ([k][m] / [k][n]); c_f32_add: C is fp32 and added to, else bf16 and
+// stored.  Leading dimensions in elements.  Returns kernels launched or a negative status.
+int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const void *B, long long ldb,
+                int b_t, void *C, long long ldc, int c_f32_add, int M, int N, int K, int *status,
+                cudaStream_t s);
+
 // Packed-metadata form of the attention predicate: m = anchor << 8 | depth.
 // (depth_k == 0 and anchor_k <= anchor_q) or (anchor_k == anchor_q and depth_k <= depth_q)
 __host__ __device__ inline bool allowed_packed(int32_t mq, int32_t mk)
