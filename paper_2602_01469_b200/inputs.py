@@ -178,6 +178,20 @@ def make_fused_rows(T: int, Hq: int, Hkv: int, D: int, seed: int):
     return tuple(out)  # qkv, dQ, dK, dV
 
 
+def make_layer_tensors(T: int, d_model: int, Hq: int, Hkv: int, D: int, seed: int):
+    """bf16 inputs of the segmented layer slice: hidden rows X [T, d_model] ~ N(0,1), the fused
+    projection weight W [(Hq + 2 Hkv) D, d_model] ~ N(0,1) / sqrt(d_model) (so that projected
+    heads have unit-variance elements), and dO [T, Hq, D] ~ N(0,1)."""
+    out = []
+    for i, (shape, std) in enumerate((((T, d_model), 1.0),
+                                      (((Hq + 2 * Hkv) * D, d_model), 1.0 / math.sqrt(d_model)),
+                                      ((T, Hq, D), 1.0))):
+        g = torch.Generator(device="cpu")
+        g.manual_seed(seed * 10 + 9 + i)
+        out.append((torch.randn(*shape, generator=g, dtype=torch.float32) * std).to(torch.bfloat16))
+    return tuple(out)  # X, W, dO
+
+
 def build_case(w: Workload, assign_fn):
     """Lays out a workload: per sequence the full grid of anchors x depths, segments from
     ``assign_fn(anchor, depth, K, boundaries) -> segment per token`` (Algorithm 1, supplied by the
