@@ -448,6 +448,60 @@ def run_rope(args, w):
     }))
 
 
+def run_gemm(args, w):
+    """The three projection products of the layer slice at the workload's shape (rows = expanded
+    tokens, d_model = args.d_model, fused width (Hq + 2 Hkv) D): a tensor-bound side line."""
+    import torch
+
+    from paper_2602_01469_b200 import binding
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    T, dm = w.total_tokens, args.d_model
+    nqkv = (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim
+    X, W, _ = inputs.make_layer_tensors(T, dm, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed)
+    X, W = X.to(dev), W.to(dev)
+    Y = torch.empty(T, nqkv, dtype=torch.bfloat16, device=dev)
+    dXa = torch.zeros(T, dm, dtype=torch.float32, device=dev)
+    dWa = torch.zeros(nqkv, dm, dtype=torch.float32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.peagle_gemm_bf16(ctx, X, dm, 0, W, dm, 0, Y, nqkv, 0, T, nqkv, dm, stream)      # Y = X W^T
+        binding.peagle_gemm_bf16(ctx, Y, nqkv, 0, W, dm, 1, dXa, dm, 1, T, dm, nqkv, stream)    # dX += Y W
+        binding.peagle_gemm_bf16(ctx, Y, nqkv, 1, X, dm, 1, dWa, dm, 1, nqkv, dm, T, stream)    # dW += Y^T X
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert binding.peagle_poll_status(ctx) == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(0) as clocks:
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    flops = 3 * 2.0 * T * nqkv * dm
+    peaks, src = load_peaks()
+    peak = float(peaks["bf16_tflops"])
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "layer projection GEMMs (forward, input grad, weight grad) TFLOP/s", "value": tf,
+        "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "rows": T, "d_model": dm, "fused_width": nqkv,
+                   "l2": "operands (%.2f GB) larger than L2, no flush" % ((T * (dm + nqkv) * 2) / 1e9)},
+        "clocks": clocks.summary(), "gpu_launches": 3 * args.steps,
+        "roofline": {"kernel": "gemm_kernel", "bound": "tensor", "achieved": tf, "peak": peak,
+                     "unit": UNIT, "frac": tf / peak, "traffic": None, "peak_source": "%s bf16_tflops (burst)" % src},
+    }))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -455,8 +509,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=inputs.HEADLINE, choices=sorted(inputs.WORKLOADS))
-    ap.add_argument("--op", default="attention", choices=["attention", "rope"],
-                    help="attention: the hot path (default); rope: the rotary prologue side line")
+    ap.add_argument("--op", default="attention", choices=["attention", "rope", "gemm"],
+                    help="attention: the hot path (default); rope: the rotary prologue side line; "
+                         "gemm: the layer slice's projection products side line")
+    ap.add_argument("--d-model", type=int, default=2880, help="hidden width for --op gemm")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "partitions"],
                     help="with --gpus N > 1: N independent replicas of the workload (default), or one "
                          "workload whose query partitions are dealt out over the ranks (dK / dV "
@@ -470,6 +526,8 @@ def main():
         run_reference(args, w)
     elif args.op == "rope":
         run_rope(args, w)
+    elif args.op == "gemm":
+        run_gemm(args, w)
     else:
         run_cuda(args, w)
 

@@ -272,6 +272,27 @@ int peagle_gemm_bf16(peagle_ctx *ctx, const void *A, int64_t lda, int a_transpos
                      int32_t M, int32_t N, int32_t K, void *stream);
 
 /*
+ * The attention half of a drafter layer, run segment by segment as Section 3.2 trains long
+ * sequences ("Our solution": one forward-backward pass per segment, gradients accumulated across
+ * the segments of a sequence; Algorithm 1 phase 3: a segment holds its own tokens and the depth-0
+ * tokens before it).  X is dev bf16 [T][d_model], the layer's input rows; W dev bf16
+ * [(n_q_heads + 2 n_kv_heads) * head_dim][d_model], the fused query | key | value projection.  For
+ * every partition in the given order: the segment's rows are projected (fused rows = X W^T) and
+ * rotated (peagle_rope_qkv_fwd); K / V of the visible tokens outside the segment's own block are
+ * projected and rotated AGAIN in this segment (they are keys only); the attention forward and
+ * backward of the partition run; the segment's dQ, dK, dV go back through the rotation and the
+ * projection, and dX, dW are summed in fp32 over the segments and rounded once at the end.
+ * Outputs: O [T][n_q_heads][head_dim] bf16 and LSE [n_q_heads][T] fp32 (rows of the partitions
+ * only), dX bf16 [T][d_model], dW bf16 like W; dO is the gradient that reaches O.  d_model a
+ * multiple of 8; rope_base > 1.  All dev; scratch of about 12 bytes per element of the fused rows
+ * is kept in the context.  Asynchronous on `stream`.
+ */
+int peagle_layer_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
+                             const peagle_partition_t *parts, int32_t nparts, const void *X,
+                             const void *W, int32_t d_model, float rope_base, const void *dO, void *O,
+                             float *LSE, void *dX, void *dW, void *stream);
+
+/*
  * Algorithm 1, host only: segment of every token.  `boundaries` is host [S+1], context-token
  * positions with boundaries[0]=0 and boundaries[S]=n (Algorithm 1's B).  Depth 0 and 1 tokens
  * go by their position anchor+depth (a position at or beyond n stays in the last segment);

@@ -27,7 +27,7 @@ EXPORTS = [
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
     "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
     "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd", "peagle_attn_partitioned_acc", "peagle_cast_grads",
-    "peagle_gemm_bf16",
+    "peagle_gemm_bf16", "peagle_layer_partitioned",
 ]
 
 
@@ -263,6 +263,14 @@ def peagle_gemm_bf16(ctx, A, lda, a_t, B, ldb, b_t, C, ldc, c_f32_add, M, N, K, 
     _check(lib().peagle_gemm_bf16(ctx.h, _ptr(A), ctypes.c_int64(lda), int(a_t), _ptr(B),
                                   ctypes.c_int64(ldb), int(b_t), _ptr(C), ctypes.c_int64(ldc),
                                   int(c_f32_add), int(M), int(N), int(K), _stream(stream)), ctx.h)
+
+
+def peagle_layer_partitioned(ctx, prob: Problem, parts, X, W, rope_base, dO, O, LSE, dX, dW, stream=None):
+    """Projection -> rotary -> attention forward and backward, one pass per segment (device tensors)."""
+    arr = _partition_array(parts)
+    _check(lib().peagle_layer_partitioned(ctx.h, prob.ref(), arr, len(parts), _ptr(X), _ptr(W),
+                                          int(X.shape[1]), ctypes.c_float(rope_base), _ptr(dO), _ptr(O),
+                                          _ptr(LSE), _ptr(dX), _ptr(dW), _stream(stream)), ctx.h)
 
 
 def peagle_assign_segments(anchor, depth, K, boundaries):

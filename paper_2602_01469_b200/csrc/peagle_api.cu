@@ -20,7 +20,7 @@ struct peagle_ctx {
     int n_sm = 0;
     EncodeTiledFn encode = nullptr;
     int *status = nullptr; // device status word
-    DevBuf plan_buf, bwd_buf, acc_buf, host_buf;
+    DevBuf plan_buf, bwd_buf, acc_buf, host_buf, layer_buf;
     int64_t launches = 0;
     char cuda_err[256] = {0};
     bool timing = false;
@@ -431,7 +431,7 @@ int peagle_destroy(peagle_ctx *ctx)
         return PEAGLE_ERR_NULL;
     cudaSetDevice(ctx->device);
     cudaDeviceSynchronize();
-    DevBuf *bufs[4] = {&ctx->plan_buf, &ctx->bwd_buf, &ctx->acc_buf, &ctx->host_buf};
+    DevBuf *bufs[5] = {&ctx->plan_buf, &ctx->bwd_buf, &ctx->acc_buf, &ctx->host_buf, &ctx->layer_buf};
     for (DevBuf *b : bufs)
         if (b->ptr)
             cudaFree(b->ptr);
@@ -817,6 +817,141 @@ int peagle_gemm_bf16(peagle_ctx *ctx, const void *A, int64_t lda, int a_transpos
     if (n < 0)
         return n;
     ctx->launches += n;
+    CK(cudaGetLastError());
+    return PEAGLE_OK;
+}
+
+int peagle_layer_partitioned(peagle_ctx *ctx, const peagle_problem_t *prob,
+                             const peagle_partition_t *parts, int32_t nparts, const void *X,
+                             const void *W, int32_t d_model, float rope_base, const void *dO, void *O,
+                             float *LSE, void *dX, void *dW, void *stream)
+{
+    if (!ctx || !X || !W || !dO || !O || !LSE || !dX || !dW || (nparts > 0 && !parts))
+        return PEAGLE_ERR_NULL;
+    int rc = check_partitioned_args(prob, parts, nparts);
+    if (rc != PEAGLE_OK)
+        return rc;
+    if (d_model < 8 || d_model % 8 != 0 || !(rope_base > 1.f))
+        return PEAGLE_ERR_BAD_SHAPE;
+    if (!aligned16(X) || !aligned16(W) || !aligned16(dO) || !aligned16(O) || !aligned16(dX) || !aligned16(dW))
+        return PEAGLE_ERR_ALIGN;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    CK(cudaSetDevice(ctx->device));
+    const size_t T = (size_t)prob->total_tokens;
+    const int Hq = prob->n_q_heads, Hkv = prob->n_kv_heads, D = prob->head_dim;
+    const size_t nq = (size_t)Hq * D, nkv = (size_t)Hkv * D, nqkv = nq + 2 * nkv, dm = (size_t)d_model;
+    if (T == 0)
+        return PEAGLE_OK;
+    // scratch: fused rows (projection output, later its gradient), the same for key-only tokens,
+    // Q K V and their gradients, fp32 sums of a segment's dK / dV, fp32 sums of dX and dW
+    auto up = [](size_t b) { return (b + 255) & ~size_t(255); };
+    const size_t b_fused = up(T * nqkv * 2), b_fkv = up(T * 2 * nkv * 2), b_q = up(T * nq * 2),
+                 b_kv = up(T * nkv * 2), b_acc = up(T * nkv * 4), b_dx = up(T * dm * 4),
+                 b_dw = up(nqkv * dm * 4);
+    rc = ensure(ctx, ctx->layer_buf, b_fused + b_fkv + 2 * b_q + 4 * b_kv + 2 * b_acc + b_dx + b_dw + 256, s);
+    if (rc != PEAGLE_OK)
+        return rc;
+    uint8_t *b = static_cast<uint8_t *>(ctx->layer_buf.ptr);
+    auto take = [&](size_t n) { uint8_t *r = b; b += n; return r; };
+    uint8_t *fused = take(b_fused), *fkv = take(b_fkv), *Qb = take(b_q), *dQb = take(b_q);
+    uint8_t *Kb = take(b_kv), *Vb = take(b_kv), *dKb = take(b_kv), *dVb = take(b_kv);
+    float *dK_acc = reinterpret_cast<float *>(take(b_acc)), *dV_acc = reinterpret_cast<float *>(take(b_acc));
+    float *dX_acc = reinterpret_cast<float *>(take(b_dx)), *dW_acc = reinterpret_cast<float *>(take(b_dw));
+    CK(cudaMemsetAsync(dX_acc, 0, T * dm * 4, s));
+    CK(cudaMemsetAsync(dW_acc, 0, nqkv * dm * 4, s));
+    const uint8_t *Xb = static_cast<const uint8_t *>(X), *Wb = static_cast<const uint8_t *>(W);
+    const uint8_t *Wkv = Wb + nq * dm * 2; // rows of W that make the key and value heads
+    auto gemm = [&](const void *A, long long lda, int a_t, const void *B, long long ldb, int b_t, void *C,
+                    long long ldc, int acc, size_t M, size_t N, size_t K) {
+        const int n = launch_gemm(ctx->encode, A, lda, a_t, B, ldb, b_t, C, ldc, acc, (int)M, (int)N, (int)K,
+                                  ctx->status, s);
+        if (n > 0)
+            ctx->launches += n;
+        return n < 0 ? n : PEAGLE_OK;
+    };
+    for (int i = 0; i < nparts; ++i) {
+        Call c;
+        rc = validate_partition(prob, &parts[i], c);
+        if (rc != PEAGLE_OK)
+            return rc;
+        const int qb = parts[i].q.begin, qe = parts[i].q.end;
+        if (qe <= qb)
+            continue;
+        // the visible tokens outside the segment's own block: keys only (Algorithm 1, phase 3)
+        int kb[2 * MAX_KRANGES], ke[2 * MAX_KRANGES], nko = 0;
+        for (int r = 0; r < c.ranges.n; ++r) {
+            const int rb = c.ranges.begin[r], re = c.ranges.end[r];
+            if (rb < qb) { kb[nko] = rb; ke[nko] = re < qb ? re : qb; ++nko; }
+            if (re > qe) { kb[nko] = rb > qe ? rb : qe; ke[nko] = re; ++nko; }
+        }
+        const size_t rows = (size_t)(qe - qb);
+        // ---- forward: projection and rotary prologue of the segment's tokens ...
+        rc = gemm(Xb + (size_t)qb * dm * 2, dm, 0, Wb, dm, 0, fused + (size_t)qb * nqkv * 2, nqkv, 0, rows, nqkv, dm);
+        if (rc != PEAGLE_OK)
+            return rc;
+        ctx->launches += launch_rope(false, fused + (size_t)qb * nqkv * 2, nullptr, nullptr, nullptr, nullptr,
+                                     Qb + (size_t)qb * nq * 2, Kb + (size_t)qb * nkv * 2, Vb + (size_t)qb * nkv * 2,
+                                     prob->anchor + qb, prob->depth + qb, (int)rows, Hq, Hkv, D, rope_base,
+                                     ctx->n_sm, s);
+        // ... and, again in this segment, K / V of the earlier depth-0 tokens it sees
+        for (int r = 0; r < nko; ++r) {
+            const size_t o = (size_t)kb[r], n = (size_t)(ke[r] - kb[r]);
+            rc = gemm(Xb + o * dm * 2, dm, 0, Wkv, dm, 0, fkv + o * 2 * nkv * 2, 2 * nkv, 0, n, 2 * nkv, dm);
+            if (rc != PEAGLE_OK)
+                return rc;
+            ctx->launches += launch_rope(false, fkv + o * 2 * nkv * 2, nullptr, nullptr, nullptr, nullptr, Qb,
+                                         Kb + o * nkv * 2, Vb + o * nkv * 2, prob->anchor + o, prob->depth + o,
+                                         (int)n, 0, Hkv, D, rope_base, ctx->n_sm, s);
+        }
+        CK(cudaGetLastError());
+        // ---- attention forward and backward of the segment; dK / dV sums of this segment only
+        for (int r = 0; r < c.ranges.n; ++r) {
+            const size_t o = (size_t)c.ranges.begin[r] * nkv, n = (size_t)(c.ranges.end[r] - c.ranges.begin[r]) * nkv;
+            CK(cudaMemsetAsync(dK_acc + o, 0, n * 4, s));
+            CK(cudaMemsetAsync(dV_acc + o, 0, n * 4, s));
+        }
+        rc = plan_call(ctx, prob, &parts[i], true, s, c);
+        if (rc != PEAGLE_OK)
+            return rc;
+        BwdArgs hand;
+        rc = bwd_scratch(ctx, prob, c, s, hand);
+        if (rc != PEAGLE_OK)
+            return rc;
+        rc = run_fwd(ctx, prob, c, Qb, Kb, Vb, O, LSE, s, dO, &hand);
+        if (rc != PEAGLE_OK)
+            return rc;
+        rc = run_bwd(ctx, prob, c, Qb, Kb, Vb, O, dO, LSE, dQb, dK_acc, dV_acc, s, true);
+        if (rc != PEAGLE_OK)
+            return rc;
+        for (int r = 0; r < c.ranges.n; ++r) {
+            const size_t o = (size_t)c.ranges.begin[r] * nkv, n = (size_t)(c.ranges.end[r] - c.ranges.begin[r]) * nkv;
+            ctx->launches += launch_cast_grads(dK_acc + o, dV_acc + o, dKb + o * 2, dVb + o * 2, n, s);
+        }
+        // ---- backward of the rotary prologue and of the projection, gradients added up over
+        // the segments (within-sequence gradient accumulation)
+        ctx->launches += launch_rope(true, nullptr, fused + (size_t)qb * nqkv * 2, dQb + (size_t)qb * nq * 2,
+                                     dKb + (size_t)qb * nkv * 2, dVb + (size_t)qb * nkv * 2, nullptr, nullptr,
+                                     nullptr, prob->anchor + qb, prob->depth + qb, (int)rows, Hq, Hkv, D,
+                                     rope_base, ctx->n_sm, s);
+        rc = gemm(fused + (size_t)qb * nqkv * 2, nqkv, 0, Wb, dm, 1, dX_acc + (size_t)qb * dm, dm, 1, rows, dm, nqkv);
+        if (rc == PEAGLE_OK)
+            rc = gemm(fused + (size_t)qb * nqkv * 2, nqkv, 1, Xb + (size_t)qb * dm * 2, dm, 1, dW_acc, dm, 1, nqkv, dm, rows);
+        for (int r = 0; rc == PEAGLE_OK && r < nko; ++r) {
+            const size_t o = (size_t)kb[r], n = (size_t)(ke[r] - kb[r]);
+            ctx->launches += launch_rope(true, nullptr, fkv + o * 2 * nkv * 2, dQb, dKb + o * nkv * 2,
+                                         dVb + o * nkv * 2, nullptr, nullptr, nullptr, prob->anchor + o,
+                                         prob->depth + o, (int)n, 0, Hkv, D, rope_base, ctx->n_sm, s);
+            rc = gemm(fkv + o * 2 * nkv * 2, 2 * nkv, 0, Wkv, dm, 1, dX_acc + o * dm, dm, 1, n, dm, 2 * nkv);
+            if (rc == PEAGLE_OK)
+                rc = gemm(fkv + o * 2 * nkv * 2, 2 * nkv, 1, Xb + o * dm * 2, dm, 1, dW_acc + nq * dm, dm, 1,
+                          2 * nkv, dm, n);
+        }
+        if (rc != PEAGLE_OK)
+            return rc;
+        CK(cudaGetLastError());
+    }
+    ctx->launches += launch_cast_one(dX_acc, dX, T * dm, s);
+    ctx->launches += launch_cast_one(dW_acc, dW, nqkv * dm, s);
     CK(cudaGetLastError());
     return PEAGLE_OK;
 }

@@ -724,6 +724,19 @@ int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cud
                      : launch_bwd_t<128>(p, a, enc, n_sm, s, ev0, ev1);
 }
 
+// One fp32 array of n elements (a multiple of 8) rounded to bf16.
+int launch_cast_one(const float *src, void *dst, size_t n, cudaStream_t s)
+{
+    const size_t n8 = n / 8;
+    if (n8 == 0)
+        return 0;
+    // the kernel takes two arrays of n8 pieces; here both are the one array, and the grid covers it
+    // once (threads past n8 in the last block repeat the first pieces with the same values)
+    cast_grads_kernel<<<(unsigned)((n8 + 255) / 256), 256, 0, s>>>(
+        src, src, static_cast<__nv_bfloat16 *>(dst), static_cast<__nv_bfloat16 *>(dst), n8);
+    return 1;
+}
+
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s)
 {

@@ -108,6 +108,7 @@ int launch_bwd(const Plan &p, const BwdArgs &a, EncodeTiledFn enc, int n_sm, cud
 int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s);
 int launch_cast_grads(const float *dK_acc, const float *dV_acc, void *dK, void *dV, size_t n,
                       cudaStream_t s);
+int launch_cast_one(const float *src, void *dst, size_t n, cudaStream_t s);
 
 // Rotary prologue (backward = false: fused row -> Q, K, V) and its backward (dQ, dK, dV -> gradient
 // of the fused row).  Returns the number of kernels launched.
