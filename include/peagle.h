@@ -315,6 +315,15 @@ int peagle_classify_tiles(peagle_ctx *ctx, const peagle_problem_t *prob,
                           const peagle_partition_t *part, uint8_t *host_out, int32_t *n_qtiles,
                           int32_t *n_ktiles);
 /*
+ * Self-test of the bounded device-side waits (no counterpart in the paper).  Every wait in the
+ * kernels gives up after a time limit, records PEAGLE_ERR_TIMEOUT in the context's status word and
+ * lets its CTA return; this call runs that path on purpose: one small CTA waits `limit_ms`
+ * milliseconds (1..1000) on a barrier that nothing arrives at.  Returns PEAGLE_OK when the kernel
+ * ran to its end; peagle_poll_status() then returns PEAGLE_ERR_TIMEOUT once, and the context stays
+ * usable.  Nothing faults or hangs.  Synchronous.
+ */
+int peagle_selftest_wait_expiry(peagle_ctx *ctx, int32_t limit_ms, void *stream);
+/*
  * The mask of one call, materialised by the device predicate: host_out[(q - q.begin) * T + k]
  * for every token k of the batch (1 = allowed and visible).  Only for q_len * T <= 2^26.
  */

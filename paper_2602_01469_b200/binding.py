@@ -27,7 +27,7 @@ EXPORTS = [
     "peagle_assign_segments", "peagle_classify_tiles", "peagle_mask_dense",
     "peagle_timing_enable", "peagle_timing_read", "peagle_attn_fwd_static",
     "peagle_rope_qkv_fwd", "peagle_rope_qkv_bwd", "peagle_attn_partitioned_acc", "peagle_cast_grads",
-    "peagle_gemm_bf16", "peagle_layer_partitioned",
+    "peagle_gemm_bf16", "peagle_layer_partitioned", "peagle_selftest_wait_expiry",
 ]
 
 
@@ -271,6 +271,11 @@ def peagle_layer_partitioned(ctx, prob: Problem, parts, X, W, rope_base, dO, O, 
     _check(lib().peagle_layer_partitioned(ctx.h, prob.ref(), arr, len(parts), _ptr(X), _ptr(W),
                                           int(X.shape[1]), ctypes.c_float(rope_base), _ptr(dO), _ptr(O),
                                           _ptr(LSE), _ptr(dX), _ptr(dW), _stream(stream)), ctx.h)
+
+
+def peagle_selftest_wait_expiry(ctx, limit_ms: int = 20, stream=None):
+    """Runs one bounded wait into its time limit; poll_status then reports TIMEOUT once."""
+    _check(lib().peagle_selftest_wait_expiry(ctx.h, int(limit_ms), _stream(stream)), ctx.h)
 
 
 def peagle_assign_segments(anchor, depth, K, boundaries):

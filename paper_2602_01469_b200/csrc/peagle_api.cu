@@ -1178,6 +1178,24 @@ int peagle_classify_tiles(peagle_ctx *ctx, const peagle_problem_t *prob,
     return PEAGLE_OK;
 }
 
+int peagle_selftest_wait_expiry(peagle_ctx *ctx, int32_t limit_ms, void *stream)
+{
+    if (!ctx)
+        return PEAGLE_ERR_NULL;
+    if (limit_ms < 1 || limit_ms > 1000)
+        return PEAGLE_ERR_BAD_SHAPE;
+    CK(cudaSetDevice(ctx->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int *flag = ctx->status + 8; // a spare word of the status allocation
+    CK(cudaMemsetAsync(flag, 0, sizeof(int), s));
+    ctx->launches += launch_wait_expiry(ctx->status, (unsigned long long)limit_ms * 1000000ull, flag, s);
+    CK(cudaGetLastError());
+    int reached = 0;
+    CK(cudaMemcpyAsync(&reached, flag, sizeof(int), cudaMemcpyDeviceToHost, s));
+    CK(cudaStreamSynchronize(s));
+    return reached == 1 ? PEAGLE_OK : PEAGLE_ERR_CUDA;
+}
+
 int peagle_mask_dense(peagle_ctx *ctx, const peagle_problem_t *prob,
                       const peagle_partition_t *part, uint8_t *host_out)
 {

@@ -35,18 +35,21 @@ int launch_bwd128_main(const CUtensorMap &tmQ, const CUtensorMap &tmdO, const CU
 //   while they turn dP^T(i) into dS^T(i):              dV(i), S^T(i+1)
 // K and V of the item sit in tensor memory as bf16 (A operands of S^T and dP^T), dS^T goes both
 // over the dP^T columns (A operand of dK) and, swizzled, to shared memory (A operand of dQ).
-// K / V tiles of the next item are prefetched into a second shared-memory stage; the items come
-// from a global cursor through a small queue.  512 threads: warps 0-7 compute, warp 8 issues
+// The K tile of the next item is prefetched into a second shared-memory stage (V has one stage: it
+// is only read when it is copied to tensor memory at the start of its item); Q / dO have three
+// stages -- with two, a stage is free only when dK of step i has run, and the reload for step i+2
+// can arrive late for S^T(i+2) (3.56 -> 3.53 ms on the headline shape, same GPU, alternating runs); the items come from
+// a global cursor through a small queue.  512 threads: warps 0-7 compute, warp 8 issues
 // MMAs, warp 9 produces, warps 12-15 drain dQ (through a swizzled fp32 tile in shared memory and
 // tiled reduce-adds) and, at the end of an item, dK / dV (global reductions from registers).
 // The drain has warps of its own because a thread with reductions in flight stalls on its next
 // proxy fence, which the compute warps need once per step for the dS^T hand-over.
 struct Bwd64Cfg {
     static constexpr int D = 64;
-    static constexpr int NSQ = 2;
+    static constexpr int NSQ = 3;
     static constexpr int TILE_BYTES = 128 * 128;
-    static constexpr int OFF_KV = 0;                              // 2 stages x (K, V)
-    static constexpr int OFF_DS = 4 * TILE_BYTES;                 // 2 panels
+    static constexpr int OFF_KV = 0;                              // K stage 0, K stage 1, V (one stage)
+    static constexpr int OFF_DS = 3 * TILE_BYTES;                 // 2 panels
     static constexpr int OFF_DQ = OFF_DS + 2 * TILE_BYTES;        // fp32 dQ tile on its way out: 2 panels of 32 columns
     static constexpr int OFF_Q = OFF_DQ + 2 * TILE_BYTES;         // ring of (Q, dO)
     static constexpr int OFF_ROW = OFF_Q + NSQ * 2 * TILE_BYTES;  // ring of (-lse2[128], -delta[128], mq[128])
@@ -235,12 +238,13 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 bool ok = true;
                 if (lane == 0) {
                     const int s = w & 1;
-                    ok = mbar_wait(BAR(B_KVEMPTY + s), ((w >> 1) & 1) ^ 1, abort_flag);
+                    ok = mbar_wait(BAR(B_KVEMPTY + s), ((w >> 1) & 1) ^ 1, abort_flag) &&
+                         (w == 0 || mbar_wait(BAR(B_KVTFULL), (w - 1) & 1, abort_flag));
                     if (ok) {
                         const int start = P.ktile[kt].x;
                         mbar_arrive_expect_tx(BAR(B_KVFULL + s), 2 * TB);
-                        tma_load_3d(sb + C::OFF_KV + (2 * s) * TB, &tmK, BAR(B_KVFULL + s), 0, g, start);
-                        tma_load_3d(sb + C::OFF_KV + (2 * s + 1) * TB, &tmV, BAR(B_KVFULL + s), 0, g, start);
+                        tma_load_3d(sb + C::OFF_KV + s * TB, &tmK, BAR(B_KVFULL + s), 0, g, start);
+                        tma_load_3d(sb + C::OFF_KV + 2 * TB, &tmV, BAR(B_KVFULL + s), 0, g, start);
                     }
                 }
                 return __all_sync(0xffffffffu, ok);
@@ -317,20 +321,19 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     break;
                 const int n_cur = P.bitems[idx / P.Hkv].w * G;
                 const int ks = w & 1;
-                const uint32_t kvo = 2 * ks * TBU;
+                const uint32_t kvo = ks * TBU;
                 // K / V of this item are in tensor memory (and its K tile in shared memory)
                 ok = mbar_wait(BAR(B_KVTFULL), w & 1, abort_flag) &&
-                     mbar_wait(BAR(B_QFULL + (it & 1)), (it >> 1) & 1, abort_flag);
+                     mbar_wait(BAR(B_QFULL + it % 3), (it / 3) & 1, abort_flag);
                 if (!ok)
                     break;
                 tc_fence_after();
-                issue_s((it & 1) * 2 * TBU);
+                issue_s((it % 3) * 2 * TBU);
                 tc_commit(BAR(B_SFULL));
-                issue_dp((it & 1) * 2 * TBU);
+                issue_dp((it % 3) * 2 * TBU);
                 tc_commit(BAR(B_DPFULL));
                 for (int i = 0; ok && i < n_cur; ++i, ++it) {
-                    const int st = it & 1, nst = st ^ 1;
-                    static_assert(NSQ == 2, "stage = step parity");
+                    const int st = it % 3, nst = (it + 1) % 3;
                     const uint32_t qo = st * 2 * TBU, nqo = nst * 2 * TBU;
                     const bool first = i == 0, last = i == n_cur - 1;
                     // ---- dV(it) once P^T(it) is in tensor memory, then S^T(it+1)
@@ -345,7 +348,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
                     if (!last) {
-                        ok = mbar_wait(BAR(B_QFULL + nst), ((it + 1) >> 1) & 1, abort_flag);
+                        ok = mbar_wait(BAR(B_QFULL + nst), ((it + 1) / 3) & 1, abort_flag);
                         if (!ok)
                             break;
                         tc_fence_after();
@@ -405,7 +408,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_KVFULL + ks), (wk.w >> 1) & 1, abort_flag));
                 if (!ok)
                     break;
-                const uint8_t *src = sp + C::OFF_KV + (2 * ks + wg) * TB + r * 128;
+                const uint8_t *src = sp + C::OFF_KV + (wg == 0 ? ks : 2) * TB + r * 128;
                 uint32_t kvw[32];
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {

@@ -96,6 +96,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int K, int seq_begin,
                 int seq_end, const RangeList &ranges, bool for_bwd, int Hkv, cudaStream_t s);
 int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s);
+// One CTA whose bounded wait runs out after limit_ns: records PEAGLE_ERR_TIMEOUT in *status.
+int launch_wait_expiry(int *status, unsigned long long limit_ns, int *reached_end, cudaStream_t s);
 
 // K1 / K2.  Return the number of kernels launched, or a negative peagle_status.
 // ev0/ev1 (may be null) are recorded on the stream right before / after the main kernel.

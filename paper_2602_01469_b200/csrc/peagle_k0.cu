@@ -11,6 +11,7 @@
 //      longest-first, and cut the backward into (key tile, query-tile chunk) work items.
 // Everything runs on the caller's stream; nothing returns to the host.
 #include "peagle_internal.h"
+#include "sm100_ptx.cuh"
 
 namespace peagle {
 
@@ -414,6 +415,38 @@ int launch_plan(const Plan &p, const int32_t *anchor, const int32_t *depth, int 
     k0_chunk_masks<<<n_ch, 128, 0, s>>>(p);
     k0_chunk_items<<<n_ch, 128, 0, s>>>(p);
     return 8;
+}
+
+// ---- self-test of the bounded waits ----------------------------------------------------------
+// One CTA waits, with the kernels' own mbar_wait, on a barrier that nothing ever arrives at; the
+// wait gives up after `limit_ns`, the CTA records PEAGLE_ERR_TIMEOUT exactly as the attention
+// kernels do, and returns.  Nothing faults and nothing spins without a limit.
+__global__ void k0_wait_expiry(int *status, unsigned long long limit_ns, int *reached_end)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ int abort_flag;
+    const uint32_t b = sm100::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        sm100::mbar_init(b, 1);
+        sm100::fence_mbar_init();
+    }
+    __syncthreads();
+    // every thread waits; the first to run out of time raises the CTA's abort flag, the others
+    // leave on seeing it
+    const bool ok = sm100::mbar_wait(b, 0, &abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (!ok || abort_flag)
+            atomicCAS(status, 0, PEAGLE_ERR_TIMEOUT);
+        *reached_end = 1;
+    }
+}
+
+int launch_wait_expiry(int *status, unsigned long long limit_ns, int *reached_end, cudaStream_t s)
+{
+    k0_wait_expiry<<<1, 64, 0, s>>>(status, limit_ns, reached_end);
+    return 1;
 }
 
 int launch_mask_dense(const Plan &p, const RangeList &ranges, uint8_t *out, cudaStream_t s)

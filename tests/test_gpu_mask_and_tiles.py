@@ -5,6 +5,7 @@ import torch
 
 from oracle import peagle_oracle as orc
 from paper_2602_01469_b200 import binding, inputs
+from tests.gpu_common import DeviceCase, check_forward
 
 pytestmark = pytest.mark.gpu
 
@@ -157,3 +158,24 @@ def test_argument_errors(ctx):
     assert status_of(lambda: binding.peagle_classify_tiles(ctx, bad, P(0, (0, 19)))) == S["BAD_SHAPE"]
     # empty query range is a no-op
     assert binding.peagle_classify_tiles(ctx, prob, P(0, (4, 4))).shape[0] == 0
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The expiry path of the kernels' waits, made to happen on the host's terms: a barrier nothing
+    arrives at, a 20 ms limit.  The kernel returns, the status word says TIMEOUT once, and the
+    context goes on working (a forward after it matches the oracle)."""
+    import time
+    c = binding.Context(0)
+    try:
+        t0 = time.perf_counter()
+        binding.peagle_selftest_wait_expiry(c, 20)
+        assert 0.015 <= time.perf_counter() - t0 < 5.0
+        assert binding.peagle_poll_status(c) == binding.STATUS["TIMEOUT"]
+        assert binding.peagle_poll_status(c) == 0                      # reported once, then cleared
+        case = DeviceCase(inputs.WORKLOADS["tiny"])
+        binding.peagle_attn_fwd(c, case.prob, case.bparts[0], case.dQ_, case.dK_, case.dV_, case.O, case.LSE)
+        assert binding.peagle_poll_status(c) == 0
+        O, LSE = case.oracle_fwd(case.parts[0])
+        check_forward(case.O.float().cpu().numpy(), case.LSE.t().cpu().numpy(), O, LSE)
+    finally:
+        c.close()
