@@ -24,7 +24,7 @@ namespace {
 
 constexpr int GT = 128;      // tile of C
 constexpr int GK = 64;       // k slab
-constexpr int G_STAGES = 4;
+constexpr int G_STAGES = 3;
 constexpr int G_TILE_BYTES = GT * GK * 2; // 16 KB per operand and stage
 constexpr int G_OFF_BAR = 2 * G_STAGES * G_TILE_BYTES;
 constexpr int G_SMEM = G_OFF_BAR + (2 * G_STAGES + 1) * 8 + 32 + 1024;
@@ -38,7 +38,7 @@ struct GemmParams {
     int *status;
 };
 
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(192, 2)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const GemmParams P)
 {
