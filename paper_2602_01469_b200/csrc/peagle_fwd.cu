@@ -2,8 +2,8 @@
 //
 // A work item is one query tile (128 rows) for two query heads of the same KV group (or one head
 // when the group size is odd), so both tiles share the K/V tiles staged in shared memory and the
-// same mask.  The kernel is persistent: one CTA per SM (a kernel that allocates tensor memory gets
-// one resident CTA per SM) draws items from a global counter, longest query tiles first, and its
+// same mask.  The kernel is persistent: one CTA per SM (it takes all of tensor memory and of the
+// register file) draws items from a global counter, longest query tiles first, and its
 // barriers, K / V ring and tensor memory carry on from item to item, so that the loads and the
 // first S product of the next item run under the last softmax and the epilogue of the current
 // one.  Roles (384 threads):
