@@ -133,6 +133,7 @@ void carve_plan(Plan &p, void *base, size_t *bytes_out)
     p.scol = c.take<uint8_t>(nq * MAX_SINGLE * BM);
     p.scs = c.take<uint8_t>(nq * MAX_SINGLE * BM);
     p.sbase = c.take<int>(nq * MAX_SINGLE);
+    p.sperm = c.take<int>(nq);
     if (bytes_out)
         *bytes_out = c.off + 256;
 }

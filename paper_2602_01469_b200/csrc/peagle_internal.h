@@ -56,6 +56,9 @@ struct Plan {
     int *sbase;            // [n_qt][MAX_SINGLE] first token of entry i's key tile
     uint8_t *scs;          // [n_qt][MAX_SINGLE][BM] what the kernels read: entry i (slots by ascending
                            // key tile) of row r is its key's column in that tile, or NO_COL
+    int *sperm;            // [n_qt] query tiles in the order the SINGLE-tile backward takes them:
+                           // by the first key tile of their SINGLE entries, so that the query
+                           // tiles that add to the same key rows run close together in time
     int *status;           // device status word
 };
 

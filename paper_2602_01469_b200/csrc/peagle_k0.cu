@@ -273,6 +273,26 @@ __global__ void k0_schedule(Plan p)
         for (int i = threadIdx.x; i < n; i += blockDim.x)
             p.qorder[i] = n - 1 - i;
     }
+    // Order of the SINGLE-tile backward: query tiles by the first token of their lowest SINGLE
+    // key tile (tiles without such entries last).  In the depth-major layout the chain tiles of
+    // one block of anchors at depths 1, 2, .. then run one after the other, and the fp32 dK / dV
+    // rows they all add to are still in L2 (one trip to memory per key row instead of one per depth).
+    __syncthreads();
+    if (n <= 8192) {
+        for (int i = threadIdx.x; i < n; i += blockDim.x)
+            cnt[i] = p.scount[i] > 0 ? p.sbase[i * MAX_SINGLE] : INT_MAX;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n; i += blockDim.x) {
+            const int ci = cnt[i];
+            int rank = 0;
+            for (int j = 0; j < n; ++j)
+                rank += (cnt[j] < ci) || (cnt[j] == ci && j < i);
+            p.sperm[rank] = i;
+        }
+    } else {
+        for (int i = threadIdx.x; i < n; i += blockDim.x)
+            p.sperm[i] = i;
+    }
 }
 
 // ---- 4c. backward work items ------------------------------------------------------------------
@@ -387,6 +407,7 @@ __global__ void k0_empty(Plan p)
     if (i < p.n_qt) {
         p.kcount[i] = 0;
         p.qorder[i] = i;
+        p.sperm[i] = i;
     }
 }
 

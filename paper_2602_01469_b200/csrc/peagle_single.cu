@@ -26,6 +26,7 @@ struct SingleParams {
     const int *scount;
     const uint8_t *scs;  // [n_qt][MAX_SINGLE][BM] key column of entry i for row r, or NO_COL
     const int *sbase;    // [n_qt][MAX_SINGLE] first token of entry i's key tile
+    const int *sperm;    // [n_qt] order in which the blocks take the query tiles
     const __nv_bfloat16 *Q, *K, *V, *O, *dO;
     const float *LSE;      // [Hq][T]
     const int32_t *meta;   // [T] packed metadata
@@ -217,7 +218,9 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
     __nv_bfloat16 *sO = sdO + (size_t)RB * row_elems;
     float *snl2 = reinterpret_cast<float *>(sO + (size_t)RB * row_elems);
     float *snd = snl2 + RB * P.Hq;
-    const int r0 = blockIdx.x * RB;
+    // blocks walk the query tiles in the order K0 chose (tiles that share key rows together); RB
+    // divides the tile height, so a block's rows lie in one tile
+    const int r0 = P.sperm[(blockIdx.x * RB) / BM] * BM + (blockIdx.x * RB) % BM;
     const int n_real = max(0, min(RB, (P.q_end - P.q_begin) - r0)); // rows of the partition
     const uint32_t bar_a = smem_u32(&bar);
     if (threadIdx.x == 0) {
@@ -299,6 +302,7 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.scount = p.scount;
     P.scs = p.scs;
     P.sbase = p.sbase;
+    P.sperm = p.sperm;
     P.Q = static_cast<const __nv_bfloat16 *>(a.Q);
     P.K = static_cast<const __nv_bfloat16 *>(a.K);
     P.V = static_cast<const __nv_bfloat16 *>(a.V);
@@ -326,9 +330,9 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     // rows per block: up to 16 units of 8 lanes within 48 KB of shared memory (the headline shape,
     // 64 heads: one row, 25 KB, 64 threads; two rows per block measured the same)
     const size_t row_bytes = (size_t)a.Hq * (3 * 64 * 2 + 8);
-    int rb = std::max(1, 16 / a.Hkv);
-    while (rb > 1 && rb * row_bytes > 48 * 1024)
-        --rb;
+    int rb = 1; // a power of two, so that it divides the tile height
+    while (2 * rb * a.Hkv <= 16 && 2 * rb * row_bytes <= 48 * 1024)
+        rb *= 2;
     const size_t smem = rb * row_bytes;
     const int threads = rb * a.Hkv * 8;
     if (threads > 128 || smem > 200 * 1024)
