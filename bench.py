@@ -33,7 +33,7 @@ UNIT = "TFLOP/s"
 # files at the time of the ncu capture; a figure whose sources have changed since reads as null.
 TRAFFIC_FILE = os.path.join(ROOT, "profiles", "traffic.json")
 CSRC = os.path.join(ROOT, "paper_2602_01469_b200", "csrc")
-BWD_KERNEL = {64: "bwd64_kernel", 128: "bwd_kernel<128>"}
+BWD_KERNEL = {64: "bwd64_kernel", 128: "bwd128_kernel"}
 FALLBACK_PEAKS = {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0}
 
 

@@ -1,4 +1,4 @@
-// Backward of the SINGLE tiles (head_dim 64): tiles in which every query row allows at most one
+// Backward of the SINGLE tiles (head_dim 64 and 128): tiles in which every query row allows at most one
 // key, such as the chain tiles of the depth-major layout.  On the tensor cores such a tile costs a
 // full 128 x 128 step for 128 useful pairs, so the pairs are done one by one on the CUDA cores.
 // For a pair (query row q of head h, key k of its KV head), with the forward's LSE and
@@ -6,7 +6,7 @@
 //   s = <Q[q,h], K[k]>,  p = exp(scale * s - LSE),  dp = <dO[q,h], V[k]>,  ds = p * (dp - Delta)
 //   dQ[q,h] += scale * ds * K[k]      dK[k] += scale * ds * Q[q,h]      dV[k] += p * dO[q,h]
 // One kernel, query-major so that no reverse (key -> queries) list is needed: eight lanes per
-// (query row, KV head) hold 8 of the 64 elements each; for every head of the group they form the
+// (query row, KV head) hold 8 elements of every 64 of the row each; for every head of the group they form the
 // row's dQ and add into per-key dK / dV sums kept in registers across the heads (one fp32 add per
 // key row at the end).  The kernel runs before the tile kernel and doubles as its preparation
 // pass: it reads O and LSE as well, writes -LSE * log2(e), -Delta and the packed metadata of
@@ -39,60 +39,63 @@ struct SingleParams {
     float scale, scale_log2;
 };
 
-// A row of 64 bf16 is spread over 8 consecutive lanes, 8 elements (one 16-byte load) per lane, so
-// that a warp reads four whole rows with every load and dot products finish with three shuffles.
+// A row of D bf16 is spread over 8 consecutive lanes: lane `sub` holds, for each 64-element panel c
+// of the row, the 8 elements 64 c + 8 sub .. + 7 (one 16-byte load per panel), so that a warp reads
+// four whole rows with every load and dot products finish with three shuffles.
+template <int CH>
 struct Chunk {
-    float v[8];
+    float v[8 * CH];
 };
-__device__ __forceinline__ Chunk unpack_chunk(const uint4 t)
+template <int CH>
+__device__ __forceinline__ Chunk<CH> unpack_chunk(const uint4 (&t)[CH])
 {
-    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
-    Chunk c;
+    Chunk<CH> c;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        c.v[2 * i] = __uint_as_float(w[i] << 16);
-        c.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    for (int j = 0; j < CH; ++j) {
+        const uint32_t w[4] = {t[j].x, t[j].y, t[j].z, t[j].w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            c.v[8 * j + 2 * i] = __uint_as_float(w[i] << 16);
+            c.v[8 * j + 2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
     }
     return c;
 }
-__device__ __forceinline__ Chunk load_chunk(const __nv_bfloat16 *row, int sub)
+template <int CH>
+__device__ __forceinline__ Chunk<CH> load_chunk(const __nv_bfloat16 *row, int sub)
 {
-    const uint4 t = reinterpret_cast<const uint4 *>(row)[sub];
-    const uint32_t w[4] = {t.x, t.y, t.z, t.w};
-    Chunk c;
+    uint4 t[CH];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        c.v[2 * i] = __uint_as_float(w[i] << 16);
-        c.v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-    return c;
+    for (int j = 0; j < CH; ++j)
+        t[j] = reinterpret_cast<const uint4 *>(row)[sub + 8 * j];
+    return unpack_chunk<CH>(t);
 }
-__device__ __forceinline__ void red_chunk(float *dst, const float (&x)[8], float f)
+// adds this lane's pieces of a row (dst = the row's first element) scaled by f
+template <int CH>
+__device__ __forceinline__ void red_chunk(float *dst, int sub, const float (&x)[8 * CH], float f)
 {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(x[0] * f),
-                 "f"(x[1] * f), "f"(x[2] * f), "f"(x[3] * f)
-                 : "memory");
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4), "f"(x[4] * f),
-                 "f"(x[5] * f), "f"(x[6] * f), "f"(x[7] * f)
-                 : "memory");
+#pragma unroll
+    for (int j = 0; j < CH; ++j) {
+        float *d = dst + 64 * j + 8 * sub;
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d), "f"(x[8 * j] * f),
+                     "f"(x[8 * j + 1] * f), "f"(x[8 * j + 2] * f), "f"(x[8 * j + 3] * f)
+                     : "memory");
+        asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(d + 4), "f"(x[8 * j + 4] * f),
+                     "f"(x[8 * j + 5] * f), "f"(x[8 * j + 6] * f), "f"(x[8 * j + 7] * f)
+                     : "memory");
+    }
 }
 
-// Unit (row r of the padded partition, KV head g) = 8 lanes; a block of 128 threads holds 16
-// units.  The kernel runs before the tile kernel and also prepares what that kernel needs per
-// (row, head): -LSE * log2(e), -Delta = -<dO, O>, the row's packed metadata, and the initial value
-// of the fp32 dQ staging row, which is this kernel's own contribution (zero for a row without
-// SINGLE keys), written with plain stores.  Keys are taken KEYS at a time so that their dK / dV
-// sums fit in registers; a row with more than KEYS keys adds its later groups with reductions.
 // Block = RB rows of the padded partition x all KV heads; unit (row, KV head g) = 8 lanes.  The
 // rows of Q, dO and O (all heads of a row are contiguous) come in by bulk copies, so that the
 // memory system sees the block's whole input at once instead of one 16-byte load per lane and
 // head; the arithmetic then reads shared memory.  The kernel runs before the tile kernel and
-// also prepares what that kernel needs per (row, head): -LSE * log2(e), -Delta = -<dO, O>, the
-// row's packed metadata, and the initial value of the fp32 dQ staging row, which is this kernel's
-// own contribution (zero for a row without SINGLE keys), written with plain stores.  Keys are
-// taken KEYS at a time so that their dK / dV sums fit in registers; a row with more than KEYS
-// keys adds its later groups with reductions.
-template <bool FIRST, int KEYS>
+// also prepares what that kernel needs per (row, head), unless the forward already left it:
+// -LSE * log2(e), -Delta = -<dO, O>, the row's packed metadata; and always the initial value of
+// the fp32 dQ staging row, which is this kernel's own contribution (zero for a row without SINGLE
+// keys), written with plain stores.  Keys are taken KEYS at a time so that their dK / dV sums fit
+// in registers; a row with more than KEYS keys adds its later groups with reductions.
+template <int D, bool FIRST, int KEYS>
 __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int ns, int sub, unsigned um,
                                             int r, int g, int qt, int rr, int G,
                                             const __nv_bfloat16 *sq, const __nv_bfloat16 *sdo,
@@ -112,32 +115,36 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
     }
     if (!any && !FIRST)
         return;
-    float dk[KEYS][8], dv[KEYS][8];
-    uint4 kp[KEYS], vp[KEYS]; // the keys' elements of this lane, packed bf16
+    constexpr int CH = D / 64, E = 8 * CH; // 16-byte pieces and elements of a row per lane
+    float dk[KEYS][E], dv[KEYS][E];
+    uint4 kp[KEYS][CH], vp[KEYS][CH]; // the keys' elements of this lane, packed bf16
 #pragma unroll
     for (int i = 0; i < KEYS; ++i) {
-        const size_t kr = ((size_t)(tok[i] >= 0 ? tok[i] : 0) * P.Hkv + g) * 64;
-        kp[i] = reinterpret_cast<const uint4 *>(P.K + kr)[sub];
-        vp[i] = reinterpret_cast<const uint4 *>(P.V + kr)[sub];
+        const size_t kr = ((size_t)(tok[i] >= 0 ? tok[i] : 0) * P.Hkv + g) * D;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
+        for (int j = 0; j < CH; ++j) {
+            kp[i][j] = reinterpret_cast<const uint4 *>(P.K + kr)[sub + 8 * j];
+            vp[i][j] = reinterpret_cast<const uint4 *>(P.V + kr)[sub + 8 * j];
+        }
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
             dk[i][e] = 0.f;
             dv[i][e] = 0.f;
         }
     }
     for (int hh = 0; hh < G; ++hh) {
         const int h = g * G + hh;
-        const Chunk q = load_chunk(sq + (size_t)h * 64, sub);
-        const Chunk dO = load_chunk(sdo + (size_t)h * 64, sub);
+        const Chunk<CH> q = load_chunk<CH>(sq + (size_t)h * D, sub);
+        const Chunk<CH> dO = load_chunk<CH>(sdo + (size_t)h * D, sub);
         float nl2, nd;
         if (FIRST && P.rows_ready) {
             nl2 = snl2[h];
             nd = snd[h];
         } else if (FIRST) {
-            const Chunk o = load_chunk(so + (size_t)h * 64, sub);
+            const Chunk<CH> o = load_chunk<CH>(so + (size_t)h * D, sub);
             float delta = 0.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e)
+            for (int e = 0; e < E; ++e)
                 delta = fmaf(dO.v[e], o.v[e], delta);
 #pragma unroll
             for (int s = 1; s < 8; s <<= 1)
@@ -156,14 +163,17 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
             nl2 = snl2[h];
             nd = snd[h];
         }
-        float dq[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        float dq[E];
+#pragma unroll
+        for (int e = 0; e < E; ++e)
+            dq[e] = 0.f;
 #pragma unroll
         for (int i = 0; i < KEYS; ++i) {
-            const Chunk k = unpack_chunk(kp[i]);
-            const Chunk v = unpack_chunk(vp[i]);
+            const Chunk<CH> k = unpack_chunk<CH>(kp[i]);
+            const Chunk<CH> v = unpack_chunk<CH>(vp[i]);
             float s = 0.f, dp = 0.f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
+            for (int e = 0; e < E; ++e) {
                 s = fmaf(q.v[e], k.v[e], s);
                 dp = fmaf(dO.v[e], v.v[e], dp);
             }
@@ -177,46 +187,56 @@ __device__ __forceinline__ void single_pass(const SingleParams &P, int i0, int n
             const float p = fast_exp2(fmaf(s, P.scale_log2, tok[i] >= 0 ? nl2 : -CUDART_INF_F)); // nl2 = -inf: p = 0
             const float ds = p * (dp + nd);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
+            for (int e = 0; e < E; ++e) {
                 dq[e] = fmaf(ds, k.v[e], dq[e]);
                 dk[i][e] = fmaf(ds, q.v[e], dk[i][e]);
                 dv[i][e] = fmaf(p, dO.v[e], dv[i][e]);
             }
         }
-        float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * 64 + sub * 8;
+        float *dst = P.dq_acc + ((size_t)r * P.Hq + h) * D;
         if (FIRST) {
-            reinterpret_cast<float4 *>(dst)[0] = make_float4(dq[0] * P.scale, dq[1] * P.scale,
-                                                             dq[2] * P.scale, dq[3] * P.scale);
-            reinterpret_cast<float4 *>(dst)[1] = make_float4(dq[4] * P.scale, dq[5] * P.scale,
-                                                             dq[6] * P.scale, dq[7] * P.scale);
+#pragma unroll
+            for (int j = 0; j < CH; ++j) {
+                float4 *d4 = reinterpret_cast<float4 *>(dst + 64 * j + 8 * sub);
+                d4[0] = make_float4(dq[8 * j] * P.scale, dq[8 * j + 1] * P.scale, dq[8 * j + 2] * P.scale,
+                                    dq[8 * j + 3] * P.scale);
+                d4[1] = make_float4(dq[8 * j + 4] * P.scale, dq[8 * j + 5] * P.scale,
+                                    dq[8 * j + 6] * P.scale, dq[8 * j + 7] * P.scale);
+            }
         } else {
-            red_chunk(dst, dq, P.scale);
+            red_chunk<CH>(dst, sub, dq, P.scale);
         }
     }
 #pragma unroll
     for (int i = 0; i < KEYS; ++i)
         if (tok[i] >= 0) {
-            const size_t kr = ((size_t)tok[i] * P.Hkv + g) * 64 + sub * 8;
-            red_chunk(P.dK_acc + kr, dk[i], P.scale);
-            red_chunk(P.dV_acc + kr, dv[i], 1.f);
+            const size_t kr = ((size_t)tok[i] * P.Hkv + g) * D;
+            red_chunk<CH>(P.dK_acc + kr, sub, dk[i], P.scale);
+            red_chunk<CH>(P.dV_acc + kr, sub, dv[i], 1.f);
         }
 }
 
-// Two keys per pass and 128 registers: the arithmetic is bound by the latency of its dependent
+// head_dim 64 runs in 128 registers: the arithmetic is bound by the latency of its dependent
 // chains (dot product, three shuffles, exp2), so more resident warps pay more than fewer passes.
-// Shared memory: [3][RB][Hq * 64] bf16 rows of Q, dO, O, then [2][RB][Hq] fp32 row values.
-__global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
+// Shared memory: [3][RB][Hq * D] bf16 rows of Q, dO, O ([2]: no O when the forward left the row
+// values), then [2][RB][Hq] fp32 row values.
+template <int D>
+__global__ void __launch_bounds__(128, D == 64 ? 4 : 2) single_bwd(const SingleParams P)
 {
+    // Two keys per pass at either head size.  Measured on 8-depth grids as the time of a step
+    // outside the two tile kernels: head_dim 64 with four keys and 168 registers 0.76 against
+    // 0.66 ms; head_dim 128 with one / two / three keys 0.45 / 0.37 / 0.40 ms.  head_dim 128 holds
+    // twice the sums per key and takes up to 255 registers.
     constexpr int KEYS = 2;
     extern __shared__ __align__(128) uint8_t smem[];
     __shared__ __align__(8) uint64_t bar;
     __shared__ int abort_flag;
     const int RB = P.rows_per_block;
-    const int row_elems = P.Hq * 64;
+    const int row_elems = P.Hq * D;
     __nv_bfloat16 *sQ = reinterpret_cast<__nv_bfloat16 *>(smem);
     __nv_bfloat16 *sdO = sQ + (size_t)RB * row_elems;
     __nv_bfloat16 *sO = sdO + (size_t)RB * row_elems;
-    float *snl2 = reinterpret_cast<float *>(sO + (size_t)RB * row_elems);
+    float *snl2 = reinterpret_cast<float *>(sO + (P.rows_ready ? 0 : (size_t)RB * row_elems));
     float *snd = snl2 + RB * P.Hq;
     // blocks walk the query tiles in the order K0 chose (tiles that share key rows together); RB
     // divides the tile height, so a block's rows lie in one tile
@@ -287,16 +307,16 @@ __global__ void __launch_bounds__(128, 4) single_bwd(const SingleParams P)
     float *rnl2 = snl2 + rl * P.Hq, *rnd = snd + rl * P.Hq;
     const int qt = r / BM, rr = r % BM;
     const int ns = min(P.scount[qt], MAX_SINGLE);
-    single_pass<true, KEYS>(P, 0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
+    single_pass<D, true, KEYS>(P, 0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
     for (int i0 = KEYS; i0 < ns; i0 += KEYS) {
         __syncwarp(um); // lane 0's row values are visible to the unit's later passes
-        single_pass<false, KEYS>(P, i0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
+        single_pass<D, false, KEYS>(P, i0, ns, sub, um, r, g, qt, rr, G, sq, sdo, so, rnl2, rnd);
     }
 }
 
 int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
 {
-    if (!p.allow_single || p.n_qt == 0 || a.D != 64)
+    if (!p.allow_single || p.n_qt == 0 || (a.D != 64 && a.D != 128))
         return 0;
     SingleParams P;
     P.scount = p.scount;
@@ -329,7 +349,7 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
     P.rows_ready = a.rows_ready ? 1 : 0;
     // rows per block: up to 16 units of 8 lanes within 48 KB of shared memory (the headline shape,
     // 64 heads: one row, 25 KB, 64 threads; two rows per block measured the same)
-    const size_t row_bytes = (size_t)a.Hq * (3 * 64 * 2 + 8);
+    const size_t row_bytes = (size_t)a.Hq * ((a.rows_ready ? 2 : 3) * a.D * 2 + 8);
     int rb = 1; // a power of two, so that it divides the tile height
     while (2 * rb * a.Hkv <= 16 && 2 * rb * row_bytes <= 48 * 1024)
         rb *= 2;
@@ -339,10 +359,10 @@ int launch_bwd_single(const Plan &p, const BwdArgs &a, cudaStream_t s)
         return PEAGLE_ERR_BAD_SHAPE;
     P.rows_per_block = rb;
     // per device, so set before every launch (host time only)
-    if (cudaFuncSetAttribute(single_bwd, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
+    void (*kern)(const SingleParams) = a.D == 64 ? single_bwd<64> : single_bwd<128>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return PEAGLE_ERR_CUDA;
-    single_bwd<<<(unsigned)((P.q_pad + rb - 1) / rb), threads, smem, s>>>(P);
+    kern<<<(unsigned)((P.q_pad + rb - 1) / rb), threads, smem, s>>>(P);
     return 1;
 }
 
