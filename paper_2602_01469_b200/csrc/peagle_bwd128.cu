@@ -8,8 +8,11 @@
 //     (its last reader of a step, dV, runs early in the step and its first reader of the next
 //     step, dP^T, late, so the reload fits between them) and a 32 KB fp32 tile through which dQ
 //     leaves in two halves by tiled reduce-adds (8-byte reductions from registers cost 0.6 of
-//     1.65 ms).  The per-row values (-LSE*log2e, -Delta, metadata) are read from global memory:
-//     the same 128 values by every thread of a column group, broadcast loads that stay in L1.
+//     1.65 ms).  -LSE*log2e and -Delta of a step's rows (1 KB) come in with its Q tile; that
+//     they fit at all takes the 1 KB usually kept as slack for aligning the tiles, so the kernel
+//     requires a 1024-byte aligned base and reports an error otherwise.  Read from global memory
+//     (broadcast loads, other rows every step) they cost 16 % of the kernel.  The packed metadata
+//     of the rows, needed by the steps that are not FULL, is still read from global memory.
 // Roles (512 threads): warps 0-7 compute (a thread owns one key lane and 64 of the 128 query
 // columns), warp 8 lane 0 issues the MMAs one step ahead (dV(i), S^T(i+1) while the compute warps
 // form dS^T(i); dK(i), dQ(i), then dP^T(i+1) while they form P^T(i+1)), warp 9 produces (TMA),
@@ -35,7 +38,13 @@ struct Bwd128Cfg {
     static constexpr int OFF_BAR = OFF_DQ + TILE_BYTES;
     static constexpr int N_BAR = 2 * NSQ + 13 + 4;               // the last four: work-queue slots
     static constexpr int OFF_MISC = OFF_BAR + N_BAR * 8;         // tensor-memory base, abort flag, queue
-    static constexpr int SMEM_BYTES = OFF_MISC + 32 + 1024;
+    // per stage of Q: -LSE*log2e and -Delta of the step's 128 query rows (2 x 512 bytes)
+    static constexpr int OFF_ROW = (OFF_MISC + 32 + 15) / 16 * 16;
+    static constexpr int ROW_BYTES = 1024;
+    // No slack for alignment is left: the kernel declares its shared memory 1024-byte aligned and
+    // leaves with an error if the base is not.
+    static constexpr int SMEM_BYTES = OFF_ROW + NSQ * ROW_BYTES;
+    static_assert(SMEM_BYTES <= 227 * 1024, "shared memory of one CTA");
     static constexpr int TM_S = 0, TM_DP = 128, TM_DQ = 128, TM_DK = 256, TM_DV = 384;
 };
 
@@ -46,10 +55,14 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 {
     using C = Bwd128Cfg;
     constexpr int D = 128, NSQ = C::NSQ, TB = C::TILE_BYTES, PB = C::PANEL_BYTES;
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t raw = smem_u32(smem_raw);
-    const uint32_t sb = (raw + 1023u) & ~1023u;
-    uint8_t *sp = smem_raw + (sb - raw);
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    const uint32_t sb = smem_u32(smem_raw);
+    uint8_t *sp = smem_raw;
+    if (sb & 1023u) { // the swizzled tiles need this alignment; nothing has been set up yet
+        if (threadIdx.x == 0)
+            atomicCAS(P.status, 0, PEAGLE_ERR_ALIGN);
+        return;
+    }
     const uint32_t bar0 = sb + C::OFF_BAR;
     auto BAR = [&](int i) { return bar0 + 8u * (uint32_t)i; };
     constexpr int B_QFULL = 0, B_QEMPTY = NSQ, B_KVFULL = 2 * NSQ, B_KVEMPTY = B_KVFULL + 1,
@@ -95,7 +108,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
     if (warp >= 12) {
         // ------------------------------------------------------------ drain (warps 12-15)
-        reg_dec<104>();
+        reg_inc<152>();
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sub = lane >> 2, cq = 2 * (lane & 3); // row inside a 16-lane load, first column
         BwdWalk wk;
@@ -145,17 +158,18 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             // partition's end are clipped by the tensor map).  The columns are released as soon
             // as the second half is in registers.
             (void)q_len;
-#pragma unroll 1
-            for (int half = 0; ok && half < 2; ++half) {
+            uint32_t o[4][32];
+#pragma unroll
+            for (int pn = 0; pn < 4; ++pn)
+                tmem_ld32(tmem + lane_base + C::TM_DQ + pn * 32, o[pn]);
+            tmem_wait_ld();
+            tc_fence_before();
+            warp_arrive(BAR(B_DQEMPTY));
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                if (!ok)
+                    break;
                 const int rw = (warp & 3) * 32 + lane; // row of the tile = tensor-memory lane
-                uint32_t o[2][32];
-                tmem_ld32(tmem + lane_base + C::TM_DQ + half * 64, o[0]);
-                tmem_ld32(tmem + lane_base + C::TM_DQ + half * 64 + 32, o[1]);
-                tmem_wait_ld();
-                if (half == 1) {
-                    tc_fence_before();
-                    warp_arrive(BAR(B_DQEMPTY));
-                }
                 if (threadIdx.x == 384)
                     bulk_wait_group_read<0>(); // the previous half has left shared memory
                 ok = bar_and(3, 128, ok);      // the four warps go on, or leave, together
@@ -167,10 +181,10 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 #pragma unroll
                     for (int c = 0; c < 8; ++c) {
                         float4 v;
-                        v.x = __uint_as_float(o[pn][4 * c]) * P.scale;
-                        v.y = __uint_as_float(o[pn][4 * c + 1]) * P.scale;
-                        v.z = __uint_as_float(o[pn][4 * c + 2]) * P.scale;
-                        v.w = __uint_as_float(o[pn][4 * c + 3]) * P.scale;
+                        v.x = __uint_as_float(o[2 * half + pn][4 * c]) * P.scale;
+                        v.y = __uint_as_float(o[2 * half + pn][4 * c + 1]) * P.scale;
+                        v.z = __uint_as_float(o[2 * half + pn][4 * c + 2]) * P.scale;
+                        v.w = __uint_as_float(o[2 * half + pn][4 * c + 3]) * P.scale;
                         *reinterpret_cast<float4 *>(dst + ((c ^ (rw & 7)) << 4)) = v;
                     }
                 }
@@ -203,7 +217,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (threadIdx.x == 384)
             bulk_wait_group<0>();
     } else if (warp >= 8) {
-        reg_dec<56>();
+        reg_dec<40>();
         if (warp == 9) {
             // -------------------------------------------------------- producer
             if (lane == 0) {
@@ -242,10 +256,14 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                 if (!ok)
                     break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(BAR(B_QFULL + st), TB);
+                    mbar_arrive_expect_tx(BAR(B_QFULL + st), TB + C::ROW_BYTES);
                     const uint32_t qa = sb + C::OFF_Q + st * TB;
                     for (int pn = 0; pn < 2; ++pn)
                         tma_load_3d(qa + pn * PB, &tmQ, BAR(B_QFULL + st), pn * 64, h, row0);
+                    const uint32_t ra = sb + C::OFF_ROW + st * C::ROW_BYTES;
+                    const size_t ri = (size_t)h * P.q_pad + (size_t)wk.qt() * BM;
+                    bulk_load(ra, P.nl2 + ri, 512, BAR(B_QFULL + st));
+                    bulk_load(ra + 512, P.nd + ri, 512, BAR(B_QFULL + st));
                 }
                 // dO has one stage: free once dV of the previous step has run
                 ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_DOEMPTY), (it & 1) ^ 1, abort_flag));
@@ -367,7 +385,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             }
         }
     } else {
-        reg_inc<176>();
+        reg_inc<160>();
         // ------------------------------------------------------------ compute (warps 0-7)
         const int wg = warp >> 2;        // half of the query columns
         const int r = threadIdx.x & 127; // key lane
@@ -385,13 +403,22 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                 mk = (r < ktile.y) ? P.meta[ktile.x + r] : META_NONE_K;
             }
             const bool full = wk.full();
-            // per-row values of this step's 64 query columns, straight from global memory
+            // per-row values of this step's 64 query columns
             const size_t rb = (size_t)wk.qt() * BM + wg * 64;
-            const float4 *nl4 = reinterpret_cast<const float4 *>(P.nl2 + (size_t)wk.head() * P.q_pad + rb);
-            const float4 *nd4 = reinterpret_cast<const float4 *>(P.nd + (size_t)wk.head() * P.q_pad + rb);
+            const uint8_t *rowv = sp + C::OFF_ROW + (it % NSQ) * C::ROW_BYTES + wg * 256;
+            const float4 *nl4 = reinterpret_cast<const float4 *>(rowv);
+            const float4 *nd4 = reinterpret_cast<const float4 *>(rowv + 512);
             const int4 *mq4 = reinterpret_cast<const int4 *>(P.mqp + rb);
-            // ---- P^T
-            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL), it & 1, abort_flag));
+            // The metadata of the next query tile is sent towards L1 now (read by the steps that are
+            // not FULL; every thread of a column group reads the same 64 values, broadcast loads)
+            {
+                int qn, hn;
+                if (lane < 2 && wk.peek(qn, hn) && qn != wk.qt())
+                    asm volatile("prefetch.global.L1 [%0];" ::"l"(P.mqp + (size_t)qn * BM + wg * 64 + lane * 32));
+            }
+            // ---- P^T (the row values arrive with the step's Q tile)
+            ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_SFULL), it & 1, abort_flag) &&
+                                             mbar_wait(BAR(B_QFULL + it % NSQ), (it / NSQ) & 1, abort_flag));
             if (!ok)
                 break;
             tc_fence_after();
@@ -402,7 +429,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             float p[64];
 #pragma unroll
             for (int c = 0; c < 64; c += 4) {
-                const float4 l = __ldg(nl4 + (c >> 2));
+                const float4 l = nl4[c >> 2];
                 p[c + 0] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 0) & 31]), P.scale_log2, l.x));
                 p[c + 1] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 1) & 31]), P.scale_log2, l.y));
                 p[c + 2] = fast_exp2(fmaf(__uint_as_float(sr[c >> 5][(c + 2) & 31]), P.scale_log2, l.z));
@@ -445,7 +472,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             }
 #pragma unroll
             for (int j = 0; j < 8; ++j) { // 16-byte chunk j = query columns 8j .. 8j+7 of this half
-                const float4 d0 = __ldg(nd4 + 2 * j), d1 = __ldg(nd4 + 2 * j + 1);
+                const float4 d0 = nd4[2 * j], d1 = nd4[2 * j + 1];
                 const int c = 8 * j;
                 uint4 v;
                 v.x = pack_bf16x2(p[c + 0] * (__uint_as_float(sr[c >> 5][(c + 0) & 31]) + d0.x),

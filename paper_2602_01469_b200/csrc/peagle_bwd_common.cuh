@@ -89,6 +89,21 @@ struct BwdWalk {
     __device__ int qt() const { return c * BWD_CQ + (__ffs(em) - 1); }
     __device__ bool full() const { return (mask >> (8 + __ffs(em) - 1)) & 1u; }
     __device__ int head() const { return g * G + hh; }
+    // (query tile, head) of the step after this one, if it belongs to the same work item
+    __device__ bool peek(int &qt_next, int &head_next) const
+    {
+        if (hh + 1 < G) {
+            qt_next = qt();
+            head_next = g * G + hh + 1;
+            return true;
+        }
+        const unsigned rest = em & (em - 1);
+        if (rest == 0)
+            return false;
+        qt_next = c * BWD_CQ + (__ffs(rest) - 1);
+        head_next = g * G;
+        return true;
+    }
     __device__ void next()
     {
         if (++hh == G) {
