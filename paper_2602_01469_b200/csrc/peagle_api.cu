@@ -36,7 +36,6 @@ namespace {
 // SINGLE tiles are taken out of the backward's tensor-core lists when the kernel that does them
 // pair by pair fits: a block of at most 16 KV heads x 8 lanes, a query row of all heads (Q, dO, O
 // and two fp32 values per head) within its shared memory.  Otherwise such tiles stay PARTIAL.
-// The forward has the pair-by-pair path for head_dim 64 only.
 bool single_tiles_ok(const peagle_problem_t *prob)
 {
     return prob->n_kv_heads <= 16 && (size_t)prob->n_q_heads * (6 * prob->head_dim + 8) <= 200 * 1024;
@@ -233,7 +232,6 @@ int plan_call(peagle_ctx *ctx, const peagle_problem_t *prob, const peagle_partit
     carve_plan(c.plan, ctx->plan_buf.ptr, nullptr);
     c.plan.status = ctx->status;
     c.plan.allow_single = single_tiles_ok(prob) ? 1 : 0;
-    c.plan.fwd_single = (c.plan.allow_single && prob->head_dim == 64) ? 1 : 0;
     if (c.plan.n_qt == 0)
         return PEAGLE_OK;
     ctx->launches += launch_plan(c.plan, prob->anchor, prob->depth, prob->K, c.seq_begin, c.seq_end,
@@ -637,7 +635,6 @@ int peagle_attn_fwd_static(int device, const peagle_problem_t *prob,
                              : reinterpret_cast<int *>(dev->scratch + STATIC_SCRATCH_BYTES - 256);
     c.plan.status = status;
     c.plan.allow_single = single_tiles_ok(prob) ? 1 : 0;
-    c.plan.fwd_single = (c.plan.allow_single && prob->head_dim == 64) ? 1 : 0;
     // The array keeps whatever the previous call left.  The status word is cleared here; the
     // plan's counters are cleared by the first K0 kernel; every other plan field this call
     // reads is written by this call's K0 kernels first.

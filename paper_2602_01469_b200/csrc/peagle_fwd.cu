@@ -23,8 +23,9 @@
 // S = Q K^T takes both operands from shared memory (K-major, 128-byte swizzle); O += P V takes
 // P from tensor memory and V from shared memory (MN-major).
 // Only tiles the classifier kept are visited; FULL tiles skip the per-element predicate; SINGLE
-// tiles (one allowed key per row, head_dim 64) pass through the same ring first and are done pair
-// by pair on the CUDA cores, their result seeding the running (m, l, O).
+// tiles (one allowed key per row) pass through the same ring first and are done pair by pair on
+// the CUDA cores, their result seeding the running (m, l, O): O in registers at head_dim 64, in
+// tensor memory at head_dim 128.
 #include <math_constants.h>
 
 #include <algorithm>
@@ -153,8 +154,8 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         it.row0 = P.q_begin + it.qt * BM;
         it.cnt = P.kcount[it.qt];
         it.klist = P.klist + (size_t)it.qt * P.n_kt;
-        // SINGLE tiles exist for head_dim 64 only; their result seeds (m, l, O) of the tile loop
-        it.n_single = (D == 64) ? min(P.scount[it.qt], MAX_SINGLE) : 0;
+        // the result of the SINGLE entries seeds (m, l, O) of the tile loop
+        it.n_single = min(P.scount[it.qt], MAX_SINGLE);
         return it;
     };
     // Roles other than the producer: index of item w, or -1 at the end (or when a wait ran out).
@@ -553,6 +554,114 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                     tmem_st32(tO + c * 32, ov);
                 }
                 tmem_wait_st(); // ordered before the first P V product by the P hand-over below
+            }
+        } else {
+            if (n_single > 0) {
+                // head_dim 128: the same pair-by-pair online softmax, but a row of O (128 fp32) does
+                // not fit beside the row of Q in registers, so O is kept in tensor memory and
+                // updated 32 columns at a time (load, scale and add, store).  Tensor-memory
+                // accesses are warp-wide, so rows without a key in an entry take part with
+                // weight 0.
+                ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_QFULL), w & 1, abort_flag));
+                uint32_t qp[64]; // the row of Q as packed bf16 pairs, panel-major
+#pragma unroll
+                for (int pn = 0; pn < 2; ++pn) {
+                    const uint8_t *qrow = sp + C::OFF_Q + x * C::TILE_BYTES + pn * C::PANEL_BYTES + r * 128;
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(qrow + ((c ^ (r & 7)) << 4));
+                        qp[32 * pn + 4 * c + 0] = v.x;
+                        qp[32 * pn + 4 * c + 1] = v.y;
+                        qp[32 * pn + 4 * c + 2] = v.z;
+                        qp[32 * pn + 4 * c + 3] = v.w;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0)
+                    mbar_arrive(BAR(B_QEMPTY)); // this warp's rows of Q are in registers
+                int col_nxt = P.scs[((size_t)qt * MAX_SINGLE) * BM + r];
+                for (int i = 0; ok && i < n_single; ++i) {
+                    const uint32_t pos = kpos + i;
+                    const int st = pos % NS, ph = (pos / NS) & 1;
+                    const int col = col_nxt;
+                    if (i + 1 < n_single) // requested one entry ahead of its use
+                        col_nxt = P.scs[((size_t)qt * MAX_SINGLE + i + 1) * BM + r];
+                    ok = __all_sync(0xffffffffu, mbar_wait(BAR(B_KFULL + st), ph, abort_flag) &&
+                                                     mbar_wait(BAR(B_VFULL + st), ph, abort_flag));
+                    if (ok) {
+                        const bool have = col != NO_COL && row_ok;
+                        const int kc = have ? col : 0;
+                        const uint8_t *krow = sp + C::OFF_K + st * C::TILE_BYTES + kc * 128;
+                        const uint8_t *vrow = sp + C::OFF_V + st * C::TILE_BYTES + kc * 128;
+                        float acc4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                        for (int pn = 0; pn < 2; ++pn) {
+#pragma unroll
+                            for (int c = 0; c < 8; ++c) {
+                                const uint4 v = *reinterpret_cast<const uint4 *>(
+                                    krow + pn * C::PANEL_BYTES + ((c ^ (kc & 7)) << 4));
+                                const uint32_t kw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const uint32_t qw = qp[32 * pn + 4 * c + k];
+                                    acc4[k] = fmaf(__uint_as_float(qw << 16), __uint_as_float(kw[k] << 16), acc4[k]);
+                                    acc4[k] = fmaf(__uint_as_float(qw & 0xffff0000u),
+                                                   __uint_as_float(kw[k] & 0xffff0000u), acc4[k]);
+                                }
+                            }
+                        }
+                        const float s2 = ((acc4[0] + acc4[1]) + (acc4[2] + acc4[3])) * P.scale_log2;
+                        float alpha = 1.f, pr = 0.f;
+                        if (have) {
+                            if (s2 > m + 8.f) { // as in the tile loop; always for the row's first key
+                                alpha = fast_exp2(m - s2); // 0 for the first key
+                                l *= alpha;
+                                m = s2;
+                            }
+                            pr = fast_exp2(s2 - m);
+                            l += pr;
+                        }
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) { // columns 32 q4 .. 32 q4 + 31 of O
+                            uint32_t ov[32];
+                            if (i > 0) {
+                                tmem_ld32(tO + q4 * 32, ov);
+                                tmem_wait_ld();
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < 32; ++e)
+                                    ov[e] = 0u;
+                            }
+                            const uint8_t *vp = vrow + (q4 >> 1) * C::PANEL_BYTES;
+#pragma unroll
+                            for (int cc = 0; cc < 4; ++cc) {
+                                const int c = (q4 & 1) * 4 + cc;
+                                const uint4 v = *reinterpret_cast<const uint4 *>(vp + ((c ^ (kc & 7)) << 4));
+                                const uint32_t vw[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+                                for (int k = 0; k < 4; ++k) {
+                                    const int e = 8 * cc + 2 * k;
+                                    ov[e] = __float_as_uint(fmaf(pr, __uint_as_float(vw[k] << 16),
+                                                                 alpha * __uint_as_float(ov[e])));
+                                    ov[e + 1] = __float_as_uint(fmaf(pr, __uint_as_float(vw[k] & 0xffff0000u),
+                                                                     alpha * __uint_as_float(ov[e + 1])));
+                                }
+                            }
+                            tmem_st32(tO + q4 * 32, ov);
+                        }
+                        tmem_wait_st(); // before the next entry loads these columns, and ordered before
+                                        // the first P V product by the P hand-over below
+                    }
+                    // every thread of this tile's four warps is done with the stage (and the four
+                    // warps leave together if a wait ran out)
+                    ok = bar_and(1 + x, 128, ok);
+                    if (!ok)
+                        break;
+                    if (r == 0) {
+                        mbar_arrive(BAR(B_KEMPTY + st));
+                        mbar_arrive(BAR(B_VEMPTY + st));
+                    }
+                }
             }
         }
         int cls_nxt = cnt > 0 ? klist[0].y >> 16 : 0;

@@ -48,8 +48,7 @@ struct Plan {
     uint16_t *cmask;       // [n_ch][n_kt] per chunk of BWD_CQ query tiles: bit b not skipped, bit 8+b FULL
     int *ccount;           // [n_ch][BWD_CQ] key tiles whose word has 1, 2, .. BWD_CQ query tiles
     int4 *bitems;          // [n_ch * n_kt] backward work items (key tile, chunk, mask word, query tiles)
-    int allow_single;      // 1: the backward of this shape takes SINGLE tiles pair by pair
-    int fwd_single;        // 1: so does the forward (head_dim 64); 0: they stay in its key lists as PARTIAL
+    int allow_single;      // 1: the kernels of this shape take SINGLE tiles pair by pair
     int *scount;           // [n_qt] SINGLE tiles found per query tile (may exceed MAX_SINGLE: clamp)
     int *skt;              // [n_qt][MAX_SINGLE] key tile of a slot
     uint8_t *sorder;       // [n_qt][MAX_SINGLE] slots by ascending key tile

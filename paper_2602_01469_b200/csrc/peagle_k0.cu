@@ -202,8 +202,8 @@ __global__ void k0_lists(Plan p)
         uint8_t c = TILE_SKIP;
         if (o < p.n_kt)
             c = p.cls[(size_t)self * p.n_kt + o];
-        if (c == TILE_SINGLE) // pair by pair in a forward that has that path, else an ordinary tile
-            c = p.fwd_single ? TILE_SKIP : TILE_PARTIAL;
+        if (c == TILE_SINGLE)
+            c = TILE_SKIP; // handled outside the tensor-core lists
         const unsigned bal = __ballot_sync(0xffffffffu, c != TILE_SKIP);
         const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
         if (lane == 0)
