@@ -44,6 +44,22 @@ int launch_bwd128_main(const CUtensorMap &tmQ, const CUtensorMap &tmdO, const CU
 // tiled reduce-adds) and, at the end of an item, dK / dV (global reductions from registers).
 // The drain has warps of its own because a thread with reductions in flight stalls on its next
 // proxy fence, which the compute warps need once per step for the dS^T hand-over.
+// Registers per thread after the roles re-split the CTA's allocation (512 threads x 128): two
+// warpgroups of compute warps, the warpgroup of the issuing / producing warps, the drain warpgroup.
+// The thread that issues the products wants its descriptors resident: with 56 (head_dim 128: 40)
+// registers for its warpgroup the compiler spilled them and re-formed them per product, and the
+// kernel was 9 (7) per cent slower than with 88.
+#ifndef BWD64_COMPUTE_REGS
+#define BWD64_COMPUTE_REGS 160
+#define BWD64_ISSUE_REGS 88
+#define BWD64_DRAIN_REGS 104
+#endif
+namespace {
+constexpr int COMPUTE_REGS = BWD64_COMPUTE_REGS, ISSUE_REGS = BWD64_ISSUE_REGS, DRAIN_REGS = BWD64_DRAIN_REGS;
+static_assert(256 * COMPUTE_REGS + 128 * ISSUE_REGS + 128 * DRAIN_REGS <= 512 * 128,
+              "the re-split must fit the launch allocation, or setmaxnreg.inc waits for ever");
+} // namespace
+
 struct Bwd64Cfg {
     static constexpr int D = 64;
     static constexpr int NSQ = 3;
@@ -121,7 +137,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
     if (warp >= 12) {
         // ------------------------------------------------------------ drain (warps 12-15)
-        reg_dec<104>();
+        reg_set<DRAIN_REGS, 128>();
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sub = lane >> 2, cq = 2 * (lane & 3); // row inside a 16-lane load, first column
         BwdWalk wk;
@@ -223,7 +239,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (threadIdx.x == 384)
             bulk_wait_group<0>();
     } else if (warp >= 8) {
-        reg_dec<56>();
+        reg_set<ISSUE_REGS, 128>();
         if (warp == 9) {
             // -------------------------------------------------------- producer
             if (lane == 0) {
@@ -384,7 +400,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
         }
     } else {
-        reg_inc<176>();
+        reg_set<COMPUTE_REGS, 128>();
         // ------------------------------------------------------------ compute (warps 0-7)
         const int wg = warp >> 2;
         const int r = threadIdx.x & 127; // key lane for S/dP/dK/dV, query row for dQ

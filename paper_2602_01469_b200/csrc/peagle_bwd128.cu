@@ -24,6 +24,22 @@
 namespace peagle {
 using namespace sm100;
 
+// Registers per thread after the roles re-split the CTA's allocation (512 threads x 128): two
+// warpgroups of compute warps, the warpgroup of the issuing / producing warps, the drain warpgroup.
+// The thread that issues the products wants its descriptors resident: with 56 (head_dim 128: 40)
+// registers for its warpgroup the compiler spilled them and re-formed them per product, and the
+// kernel was 9 (7) per cent slower than with 88.
+#ifndef BWD128_COMPUTE_REGS
+#define BWD128_COMPUTE_REGS 144
+#define BWD128_ISSUE_REGS 88
+#define BWD128_DRAIN_REGS 136
+#endif
+namespace {
+constexpr int COMPUTE_REGS = BWD128_COMPUTE_REGS, ISSUE_REGS = BWD128_ISSUE_REGS, DRAIN_REGS = BWD128_DRAIN_REGS;
+static_assert(256 * COMPUTE_REGS + 128 * ISSUE_REGS + 128 * DRAIN_REGS <= 512 * 128,
+              "the re-split must fit the launch allocation, or setmaxnreg.inc waits for ever");
+} // namespace
+
 struct Bwd128Cfg {
     static constexpr int D = 128;
     static constexpr int NSQ = 2;
@@ -108,7 +124,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
 
     if (warp >= 12) {
         // ------------------------------------------------------------ drain (warps 12-15)
-        reg_inc<152>();
+        reg_set<DRAIN_REGS, 128>();
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const int sub = lane >> 2, cq = 2 * (lane & 3); // row inside a 16-lane load, first column
         BwdWalk wk;
@@ -217,7 +233,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
         if (threadIdx.x == 384)
             bulk_wait_group<0>();
     } else if (warp >= 8) {
-        reg_dec<40>();
+        reg_set<ISSUE_REGS, 128>();
         if (warp == 9) {
             // -------------------------------------------------------- producer
             if (lane == 0) {
@@ -385,7 +401,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             }
         }
     } else {
-        reg_inc<160>();
+        reg_set<COMPUTE_REGS, 128>();
         // ------------------------------------------------------------ compute (warps 0-7)
         const int wg = warp >> 2;        // half of the query columns
         const int r = threadIdx.x & 127; // key lane

@@ -342,6 +342,18 @@ __device__ __forceinline__ void reg_dec()
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
 }
 
+// Sets the warpgroup's register count to N from the LAUNCH value every warp starts with, by the
+// instruction that fits (an .inc below the current count, or a .dec above it, is illegal).
+template <int N, int LAUNCH>
+__device__ __forceinline__ void reg_set()
+{
+    static_assert(N % 8 == 0 && N >= 24 && N <= 256, "setmaxnreg takes a multiple of 8 in [24, 256]");
+    if constexpr (N > LAUNCH)
+        reg_inc<N>();
+    else if constexpr (N < LAUNCH)
+        reg_dec<N>();
+}
+
 // ------------------------------------------------------------------ packed fp32 pairs
 // (d0, d1) = (a0, a1) * (b0, b1) + (c0, c1) in one instruction.
 __device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b0, float b1,
