@@ -57,7 +57,8 @@ typedef enum peagle_status {
     PEAGLE_ERR_TIMEOUT = -7,          /* a bounded device-side wait expired (device-side check) */
     PEAGLE_ERR_TOO_LARGE = -8,        /* request exceeds a documented limit */
     PEAGLE_ERR_CUDA = -9,             /* a CUDA runtime/driver call failed; see peagle_last_cuda_error */
-    PEAGLE_ERR_ALIGN = -10            /* a tensor base address is not 16-byte aligned */
+    PEAGLE_ERR_ALIGN = -10            /* a tensor base address is not 16-byte aligned; or (device-side check, head_dim 128
+                                         backward) the kernel's shared memory does not start on a 1024-byte boundary */
 } peagle_status;
 
 typedef struct peagle_ctx peagle_ctx; /* opaque: device id, scratch memory, device status word */
