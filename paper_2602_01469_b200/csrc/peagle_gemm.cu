@@ -9,11 +9,12 @@
 //   forward      Y  = X W^T      A = X  [rows][d_in]  K-major,  B = W [d_out][d_in] K-major
 //   input grad   dX = dY W       A = dY [rows][d_out] K-major,  B = W [d_out][d_in] MN-major (k = d_out)
 //   weight grad  dW = dY^T X     A = dY [rows][d_out] MN-major, B = X [rows][d_in]  MN-major (k = rows)
-// One CTA computes one 128 x 128 tile of C: warp 0 loads 64-wide k slabs of A and B by TMA into a
-// ring of stages (128-byte swizzle), warp 1 lane 0 issues tcgen05.mma (four k = 16 products per
-// slab) and releases the stages by commits, warps 2-5 read the accumulator when the last commit
-// arrives and either store bf16 rows or add into an fp32 C (tiles of one launch are disjoint and
-// launches on a stream are ordered, so the addition is a plain load-add-store).
+// Persistent CTAs take 128 x 128 or 128 x 256 tiles of C in turn: warp 0 loads 64-wide k slabs of A
+// and B by TMA into a ring of stages (128-byte swizzle), warp 1 lane 0 issues tcgen05.mma (four
+// k = 16 products per slab) into one of two accumulators in tensor memory and releases the stages
+// by commits, warps 2-5 read an accumulator when its last commit arrives, hand it back as soon as
+// it is in registers, and either store bf16 rows or add into an fp32 C (tiles of one launch are
+// disjoint and launches on a stream are ordered, so the addition is a plain load-add-store).
 #include "peagle_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -22,12 +23,23 @@ using namespace sm100;
 
 namespace {
 
-constexpr int GT = 128;      // tile of C
+constexpr int GT = 128;      // rows of a tile of C
 constexpr int GK = 64;       // k slab
-constexpr int G_STAGES = 3;
-constexpr int G_TILE_BYTES = GT * GK * 2; // 16 KB per operand and stage
-constexpr int G_OFF_BAR = 2 * G_STAGES * G_TILE_BYTES;
-constexpr int G_SMEM = G_OFF_BAR + (2 * G_STAGES + 1) * 8 + 32 + 1024;
+constexpr int G_TILE_BYTES = GT * GK * 2; // 16 KB: 128 rows of an operand, one stage
+// A tile of C is 128 x NT.  NT = 128: three stages, two CTAs per SM (one's epilogue under the
+// other's products).  NT = 256: the products are twice as wide, so the A operand and the
+// instruction stream are shared by twice the work and a product moves 12 instead of 16 KB of
+// shared memory per 128 columns; four stages of 48 KB, one CTA per SM.
+template <int NT>
+struct GemmCfg {
+    static constexpr int STAGES = NT == 128 ? 3 : 4;
+    static constexpr int B_BYTES = (NT / GT) * G_TILE_BYTES;
+    static constexpr int STAGE_BYTES = G_TILE_BYTES + B_BYTES;
+    static constexpr int OFF_BAR = STAGES * STAGE_BYTES;
+    static constexpr int N_BAR = 2 * STAGES + 4; // + two accumulators: full, empty
+    static constexpr int SMEM = OFF_BAR + N_BAR * 8 + 32 + 1024;
+    static constexpr int CTAS = NT == 128 ? 2 : 1;
+};
 
 struct GemmParams {
     int M, N, K;
@@ -38,7 +50,8 @@ struct GemmParams {
     int *status;
 };
 
-__global__ void __launch_bounds__(192, 2)
+template <int NT>
+__global__ void __launch_bounds__(192, GemmCfg<NT>::CTAS)
 gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
             const GemmParams P)
 {
@@ -46,15 +59,23 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t sb = (raw + 1023u) & ~1023u;
     uint8_t *sp = smem_raw + (sb - raw);
+    using C = GemmCfg<NT>;
+    constexpr int G_STAGES = C::STAGES, G_OFF_BAR = C::OFF_BAR;
     const uint32_t bar0 = sb + G_OFF_BAR;
     auto FULL = [&](int s) { return bar0 + 8u * (uint32_t)s; };
     auto EMPTY = [&](int s) { return bar0 + 8u * (uint32_t)(G_STAGES + s); };
-    const uint32_t ACC = bar0 + 8u * (2 * G_STAGES);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + G_OFF_BAR + (2 * G_STAGES + 1) * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + G_OFF_BAR + (2 * G_STAGES + 1) * 8 + 4);
+    auto ACCFULL = [&](int b) { return bar0 + 8u * (uint32_t)(2 * G_STAGES + b); };
+    auto ACCEMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * G_STAGES + 2 + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + G_OFF_BAR + C::N_BAR * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + G_OFF_BAR + C::N_BAR * 8 + 4);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m0 = blockIdx.y * GT, n0 = blockIdx.x * GT;
     const int n_k = (P.K + GK - 1) / GK;
+    // The CTA is persistent: it takes the tiles blockIdx.x, + gridDim.x, ... in row-major order of C
+    // (CTAs running together then share a few row blocks of A, and B stays in L2), with two
+    // accumulators in tensor memory so that the epilogue of a tile runs under the next one's
+    // products.
+    const int tiles_n = (P.N + NT - 1) / NT;
+    const int n_tiles = tiles_n * ((P.M + GT - 1) / GT);
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
@@ -62,11 +83,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             mbar_init(FULL(s), 1);
             mbar_init(EMPTY(s), 1);
         }
-        mbar_init(ACC, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(ACCFULL(b), 1);
+            mbar_init(ACCEMPTY(b), 4); // one arrival per epilogue warp
+        }
         fence_mbar_init();
     }
     if (warp == 1) {
-        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), 128);
+        tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_slot)), 2 * NT);
         tmem_relinquish();
     }
     tc_fence_before();
@@ -79,12 +103,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
         if (lane == 0) {
             tma_prefetch_desc(&tmA);
             tma_prefetch_desc(&tmB);
-            for (int i = 0; i < n_k; ++i) {
-                const int s = i % G_STAGES;
-                if (!mbar_wait(EMPTY(s), ((i / G_STAGES) & 1) ^ 1, abort_flag))
+            bool live = true;
+            int it = 0; // k slabs loaded so far, over all tiles of this CTA
+            for (int t = blockIdx.x; live && t < n_tiles; t += gridDim.x) {
+            const int m0 = (t / tiles_n) * GT, n0 = (t % tiles_n) * NT;
+            for (int i = 0; i < n_k; ++i, ++it) {
+                const int s = it % G_STAGES;
+                if (!mbar_wait(EMPTY(s), ((it / G_STAGES) & 1) ^ 1, abort_flag)) {
+                    live = false;
                     break;
-                mbar_arrive_expect_tx(FULL(s), 2 * G_TILE_BYTES);
-                const uint32_t a = sb + s * 2 * G_TILE_BYTES, b = a + G_TILE_BYTES;
+                }
+                mbar_arrive_expect_tx(FULL(s), C::STAGE_BYTES);
+                const uint32_t a = sb + s * C::STAGE_BYTES, b = a + G_TILE_BYTES;
                 const int k0 = i * GK;
                 if (!P.a_t) {
                     tma_load_2d(a, &tmA, FULL(s), k0, m0); // [128 m][64 k]
@@ -93,51 +123,71 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                     tma_load_2d(a + G_TILE_BYTES / 2, &tmA, FULL(s), m0 + 64, k0);
                 }
                 if (!P.b_t) {
-                    tma_load_2d(b, &tmB, FULL(s), k0, n0);
-                } else {
-                    tma_load_2d(b, &tmB, FULL(s), n0, k0);
-                    tma_load_2d(b + G_TILE_BYTES / 2, &tmB, FULL(s), n0 + 64, k0);
+                    tma_load_2d(b, &tmB, FULL(s), k0, n0); // [NT n][64 k]
+                } else {                                    // NT / 64 panels [64 k][64 n]
+#pragma unroll
+                    for (int pn = 0; pn < NT / 64; ++pn)
+                        tma_load_2d(b + pn * (G_TILE_BYTES / 2), &tmB, FULL(s), n0 + 64 * pn, k0);
                 }
+            }
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------ MMA issue
         if (lane == 0) {
-            const uint32_t idesc = idesc_bf16_f32(GT, GT, P.a_t, P.b_t);
+            const uint32_t idesc = idesc_bf16_f32(GT, NT, P.a_t, P.b_t);
             // K-major: a k = 16 slice is 32 bytes further inside the 128-byte rows; MN-major: 16
             // rows (2,048 bytes) further, the second 64-wide panel half a tile on
             const uint32_t a_step = P.a_t ? 128u : 2u, b_step = P.b_t ? 128u : 2u;
             bool ok = true;
-            for (int i = 0; ok && i < n_k; ++i) {
-                const int s = i % G_STAGES;
-                ok = mbar_wait(FULL(s), (i / G_STAGES) & 1, abort_flag);
+            int it = 0, j = 0; // k slabs and tiles done so far
+            for (int t = blockIdx.x; ok && t < n_tiles; t += gridDim.x, ++j) {
+            const int buf = j & 1;
+            // the epilogue has read this accumulator's previous tile
+            ok = mbar_wait(ACCEMPTY(buf), ((j >> 1) & 1) ^ 1, abort_flag);
+            if (!ok)
+                break;
+            tc_fence_after();
+            for (int i = 0; ok && i < n_k; ++i, ++it) {
+                const int s = it % G_STAGES;
+                ok = mbar_wait(FULL(s), (it / G_STAGES) & 1, abort_flag);
                 if (!ok)
                     break;
                 tc_fence_after();
-                const uint32_t a = sb + s * 2 * G_TILE_BYTES, b = a + G_TILE_BYTES;
+                const uint32_t a = sb + s * C::STAGE_BYTES, b = a + G_TILE_BYTES;
                 const uint32_t a_lo = desc_lo_sw128(a, P.a_t ? G_TILE_BYTES / 2 : 16);
                 const uint32_t b_lo = desc_lo_sw128(b, P.b_t ? G_TILE_BYTES / 2 : 16);
 #pragma unroll
                 for (int k = 0; k < GK / 16; ++k)
-                    mma_ss_lo(tmem, a_lo + k * a_step, b_lo + k * b_step, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    mma_ss_lo(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
+                              (i > 0 || k > 0) ? 1u : 0u);
                 tc_commit(EMPTY(s));
             }
             if (ok)
-                tc_commit(ACC);
+                tc_commit(ACCFULL(buf));
+            }
         }
     } else {
         // ------------------------------------------------------------ epilogue (warps 2-5)
         const int q = warp & 3; // tensor-memory lane quarter this warp may read
-        const int m = m0 + q * 32 + lane;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(ACC, 0, abort_flag));
-        if (ok) {
+        int j = 0;
+        for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++j) {
+            const int buf = j & 1;
+            const int m0 = (t / tiles_n) * GT, n0 = (t % tiles_n) * NT;
+            const int m = m0 + q * 32 + lane;
+            if (!__all_sync(0xffffffffu, mbar_wait(ACCFULL(buf), (j >> 1) & 1, abort_flag)))
+                break;
             tc_fence_after();
-            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16);
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + buf * NT;
 #pragma unroll 1
-            for (int c = 0; c < GT / 32; ++c) {
+            for (int c = 0; c < NT / 32; ++c) {
                 uint32_t o[32];
                 tmem_ld32(trow + c * 32, o);
                 tmem_wait_ld();
+                if (c == NT / 32 - 1) { // the accumulator is in registers: the next tile may take it
+                    tc_fence_before();
+                    warp_arrive(ACCEMPTY(buf));
+                }
                 const int n = n0 + c * 32;
                 if (m >= P.M)
                     continue;
@@ -186,7 +236,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        tmem_dealloc(tmem, 128);
+        tmem_dealloc(tmem, 2 * NT);
     }
 }
 
@@ -219,7 +269,10 @@ int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const 
     CUtensorMap tmA, tmB;
     // K-major operand [R][K]: boxes of 64 k x 128 rows; transposed [K][R]: boxes of 64 r x 64 k
     const int ra = a_t ? matrix_map(enc, &tmA, A, K, M, lda, 64, 64) : matrix_map(enc, &tmA, A, M, K, lda, 64, GT);
-    const int rb = b_t ? matrix_map(enc, &tmB, B, K, N, ldb, 64, 64) : matrix_map(enc, &tmB, B, N, K, ldb, 64, GT);
+    // wide tiles where they do not waste much of the last column of tiles
+    const bool wide = N >= 1024 && ((N + 255) / 256) * 256 <= N + N / 8;
+    const int NT = wide ? 256 : 128;
+    const int rb = b_t ? matrix_map(enc, &tmB, B, K, N, ldb, 64, 64) : matrix_map(enc, &tmB, B, N, K, ldb, 64, NT);
     if (ra || rb)
         return PEAGLE_ERR_CUDA;
     GemmParams P;
@@ -232,10 +285,24 @@ int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const 
     P.C = C;
     P.ldc = ldc;
     P.status = status;
-    if (cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, G_SMEM) != cudaSuccess)
+    int dev = 0, n_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return PEAGLE_ERR_CUDA;
-    dim3 grid((unsigned)((N + GT - 1) / GT), (unsigned)((M + GT - 1) / GT));
-    gemm_kernel<<<grid, 192, G_SMEM, s>>>(tmA, tmB, P);
+    const long long n_tiles = (long long)((N + NT - 1) / NT) * ((M + GT - 1) / GT);
+    const long long resident = (long long)n_sm * (wide ? GemmCfg<256>::CTAS : GemmCfg<128>::CTAS);
+    const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
+    if (wide) {
+        if (cudaFuncSetAttribute(gemm_kernel<256>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 GemmCfg<256>::SMEM) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        gemm_kernel<256><<<grid, 192, GemmCfg<256>::SMEM, s>>>(tmA, tmB, P);
+    } else {
+        if (cudaFuncSetAttribute(gemm_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 GemmCfg<128>::SMEM) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        gemm_kernel<128><<<grid, 192, GemmCfg<128>::SMEM, s>>>(tmA, tmB, P);
+    }
     return 1;
 }
 
