@@ -240,6 +240,212 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
     }
 }
 
+// ---- the same product by pairs of CTAs (a cluster of two, tcgen05 cta_group::2) -------------
+// A pair takes 256 x 256 tiles of C: each CTA loads its own 128 rows of A and its own half (128
+// of the 256 columns) of B, one thread of the pair's first CTA issues M = 256 products that read
+// both CTAs' shared memory and write both CTAs' tensor memory, and each CTA's epilogue warps read
+// their own 128 rows of the accumulator.  Per 128 x 256 of C a CTA now stages 32 KB per k slab
+// instead of 48.  No load is multicast: every CTA's TMA writes its own shared memory; the bytes
+// of both CTAs are counted on the first CTA's barrier of the stage (the cta_group::2 form of the
+// load lets the second CTA name it), and stages and accumulators are handed back to both CTAs by
+// multicast commits.
+struct Gemm2Cfg {
+    static constexpr int NT = 256;
+    static constexpr int STAGES = 6;
+    static constexpr int STAGE_BYTES = 2 * G_TILE_BYTES; // A: 128 m x 64 k, B half: 128 n x 64 k
+    static constexpr int OFF_BAR = STAGES * STAGE_BYTES;
+    static constexpr int N_BAR = 2 * STAGES + 4; // full, empty per stage; accumulator full / empty x 2
+    static constexpr int SMEM = OFF_BAR + N_BAR * 8 + 32 + 1024;
+};
+
+__global__ void __launch_bounds__(192, 1)
+gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+             const GemmParams P)
+{
+    using C = Gemm2Cfg;
+    constexpr int NT = C::NT, ST = C::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t sb = (raw + 1023u) & ~1023u; // the same offset in both CTAs of the pair
+    uint8_t *sp = smem_raw + (sb - raw);
+    const uint32_t bar0 = sb + C::OFF_BAR;
+    auto FULL = [&](int s) { return bar0 + 8u * (uint32_t)s; };
+    auto EMPTY = [&](int s) { return bar0 + 8u * (uint32_t)(ST + s); };
+    auto ACCFULL = [&](int b) { return bar0 + 8u * (uint32_t)(2 * ST + b); };
+    auto ACCEMPTY = [&](int b) { return bar0 + 8u * (uint32_t)(2 * ST + 2 + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(sp + C::OFF_BAR + C::N_BAR * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(sp + C::OFF_BAR + C::N_BAR * 8 + 4);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank(); // 0: issues the products
+    const int n_k = (P.K + GK - 1) / GK;
+    const int tiles_n = (P.N + NT - 1) / NT;
+    const int n_tiles = tiles_n * ((P.M + 2 * GT - 1) / (2 * GT));
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < ST; ++s) {
+            mbar_init(FULL(s), 1);  // used in the first CTA: one arrival, the bytes of both CTAs
+            mbar_init(EMPTY(s), 1); // one multicast commit
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(ACCFULL(b), 1);
+            mbar_init(ACCEMPTY(b), 8); // used in the first CTA: four epilogue warps of each CTA
+        }
+        fence_mbar_init();
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(smem_u32(const_cast<uint32_t *>(tmem_slot)), 2 * NT);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all(); // both CTAs' barriers exist before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+
+    if (warp == 0) {
+        // ------------------------------------------------------------ producer (each CTA its own)
+        if (lane == 0) {
+            tma_prefetch_desc(&tmA);
+            tma_prefetch_desc(&tmB);
+            bool live = true;
+            int it = 0;
+            for (int t = pair; live && t < n_tiles; t += n_pairs) {
+                const int m0 = (t / tiles_n) * 2 * GT + (int)rank * GT;
+                const int nb = (t % tiles_n) * NT + (int)rank * (NT / 2); // this CTA's half of B
+                for (int i = 0; i < n_k; ++i, ++it) {
+                    const int s = it % ST;
+                    if (!mbar_wait_cluster(EMPTY(s), ((it / ST) & 1) ^ 1, abort_flag)) {
+                        live = false;
+                        break;
+                    }
+                    if (rank == 0)
+                        mbar_arrive_expect_tx(FULL(s), 2 * C::STAGE_BYTES); // both CTAs' slabs
+                    const uint32_t full = cluster_map(FULL(s), 0);
+                    const uint32_t a = sb + s * C::STAGE_BYTES, b = a + G_TILE_BYTES;
+                    const int k0 = i * GK;
+                    if (!P.a_t) {
+                        tma_load_2d_pair(a, &tmA, full, k0, m0);
+                    } else {
+                        tma_load_2d_pair(a, &tmA, full, m0, k0);
+                        tma_load_2d_pair(a + G_TILE_BYTES / 2, &tmA, full, m0 + 64, k0);
+                    }
+                    if (!P.b_t) {
+                        tma_load_2d_pair(b, &tmB, full, k0, nb);
+                    } else {
+                        tma_load_2d_pair(b, &tmB, full, nb, k0);
+                        tma_load_2d_pair(b + G_TILE_BYTES / 2, &tmB, full, nb + 64, k0);
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // ---------------------------------------- first CTA: the pair's products
+            const uint32_t idesc = idesc_bf16_f32(2 * GT, NT, P.a_t, P.b_t);
+            const uint32_t a_step = P.a_t ? 128u : 2u, b_step = P.b_t ? 128u : 2u;
+            bool ok = true;
+            int it = 0, j = 0;
+            for (int t = pair; ok && t < n_tiles; t += n_pairs, ++j) {
+                const int buf = j & 1;
+                ok = mbar_wait_cluster(ACCEMPTY(buf), ((j >> 1) & 1) ^ 1, abort_flag);
+                if (!ok)
+                    break;
+                tc_fence_after();
+                for (int i = 0; ok && i < n_k; ++i, ++it) {
+                    const int s = it % ST;
+                    ok = mbar_wait_cluster(FULL(s), (it / ST) & 1, abort_flag);
+                    if (!ok)
+                        break;
+                    tc_fence_after();
+                    const uint32_t a = sb + s * C::STAGE_BYTES, b = a + G_TILE_BYTES;
+                    const uint32_t a_lo = desc_lo_sw128(a, P.a_t ? G_TILE_BYTES / 2 : 16);
+                    const uint32_t b_lo = desc_lo_sw128(b, P.b_t ? G_TILE_BYTES / 2 : 16);
+#pragma unroll
+                    for (int k = 0; k < GK / 16; ++k)
+                        mma_ss_lo_pair(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
+                                       (i > 0 || k > 0) ? 1u : 0u);
+                    tc_commit_pair(EMPTY(s));
+                }
+                if (ok)
+                    tc_commit_pair(ACCFULL(buf));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2-5, each CTA)
+        const int q = warp & 3;
+        int j = 0;
+        for (int t = pair; t < n_tiles; t += n_pairs, ++j) {
+            const int buf = j & 1;
+            const int m = (t / tiles_n) * 2 * GT + (int)rank * GT + q * 32 + lane;
+            const int n0 = (t % tiles_n) * NT;
+            if (!__all_sync(0xffffffffu, mbar_wait_cluster(ACCFULL(buf), (j >> 1) & 1, abort_flag)))
+                break;
+            tc_fence_after();
+            const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + buf * NT;
+#pragma unroll 1
+            for (int c = 0; c < NT / 32; ++c) {
+                uint32_t o[32];
+                tmem_ld32(trow + c * 32, o);
+                tmem_wait_ld();
+                if (c == NT / 32 - 1) { // in registers: the first CTA may reuse the accumulator
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0)
+                        mbar_arrive_remote(ACCEMPTY(buf), 0);
+                }
+                const int n = n0 + c * 32;
+                if (m >= P.M)
+                    continue;
+                if (!P.c_f32_add) {
+                    __nv_bfloat16 *dst = static_cast<__nv_bfloat16 *>(P.C) + (size_t)m * P.ldc + n;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 8) {
+                        if (n + i < P.N) {
+                            uint4 v;
+                            v.x = pack_bf16x2(__uint_as_float(o[i + 0]), __uint_as_float(o[i + 1]));
+                            v.y = pack_bf16x2(__uint_as_float(o[i + 2]), __uint_as_float(o[i + 3]));
+                            v.z = pack_bf16x2(__uint_as_float(o[i + 4]), __uint_as_float(o[i + 5]));
+                            v.w = pack_bf16x2(__uint_as_float(o[i + 6]), __uint_as_float(o[i + 7]));
+                            *reinterpret_cast<uint4 *>(dst + i) = v;
+                        }
+                    }
+                } else {
+                    float *dst = static_cast<float *>(P.C) + (size_t)m * P.ldc + n;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        if (n + i < P.N) {
+                            float4 v = *reinterpret_cast<float4 *>(dst + i);
+                            v.x += __uint_as_float(o[i + 0]);
+                            v.y += __uint_as_float(o[i + 1]);
+                            v.z += __uint_as_float(o[i + 2]);
+                            v.w += __uint_as_float(o[i + 3]);
+                            *reinterpret_cast<float4 *>(dst + i) = v;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------------------------------------ teardown
+    // Both CTAs meet before either frees tensor memory or leaves: the first CTA's products and
+    // commits reach into the second, and remote arrivals into the first.  Every wait above is
+    // bounded, so both get here.
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (*abort_flag && threadIdx.x == 0)
+        atomicCAS(P.status, 0, PEAGLE_ERR_TIMEOUT);
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc_pair(tmem, 2 * NT);
+    }
+}
+
 // Tensor map of a row-major bf16 matrix [rows][cols] with leading dimension ld (elements).
 int matrix_map(EncodeTiledFn enc, CUtensorMap *m, const void *base, long long rows, long long cols,
                long long ld, int box_cols, int box_rows)
@@ -272,7 +478,13 @@ int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const 
     // wide tiles where they do not waste much of the last column of tiles
     const bool wide = N >= 1024 && ((N + 255) / 256) * 256 <= N + N / 8;
     const int NT = wide ? 256 : 128;
-    const int rb = b_t ? matrix_map(enc, &tmB, B, K, N, ldb, 64, 64) : matrix_map(enc, &tmB, B, N, K, ldb, 64, NT);
+    // pairs of CTAs where there are at least two row blocks to pair
+#ifndef PEAGLE_GEMM_PAIRS
+#define PEAGLE_GEMM_PAIRS 1
+#endif
+    const bool pairs = PEAGLE_GEMM_PAIRS && wide && M > GT;
+    const int rb = b_t ? matrix_map(enc, &tmB, B, K, N, ldb, 64, 64)
+                       : matrix_map(enc, &tmB, B, N, K, ldb, 64, pairs ? GT : NT);
     if (ra || rb)
         return PEAGLE_ERR_CUDA;
     GemmParams P;
@@ -289,6 +501,32 @@ int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const 
     if (cudaGetDevice(&dev) != cudaSuccess ||
         cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
         return PEAGLE_ERR_CUDA;
+    if (pairs) {
+        if (cudaFuncSetAttribute(gemm2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 Gemm2Cfg::SMEM) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = 2;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        cfg.blockDim = dim3(192);
+        cfg.dynamicSmemBytes = Gemm2Cfg::SMEM;
+        cfg.stream = s;
+        cfg.gridDim = dim3((unsigned)(n_sm & ~1));
+        int fit = 0; // pairs that can be resident at once
+        if (cudaOccupancyMaxActiveClusters(&fit, gemm2_kernel, &cfg) != cudaSuccess || fit < 1)
+            return PEAGLE_ERR_CUDA;
+        const long long tiles2 = (long long)((N + 255) / 256) * ((M + 255) / 256);
+        const long long n_pairs = tiles2 < fit ? tiles2 : fit;
+        cfg.gridDim = dim3((unsigned)(2 * n_pairs));
+        if (cudaLaunchKernelEx(&cfg, gemm2_kernel, tmA, tmB, P) != cudaSuccess)
+            return PEAGLE_ERR_CUDA;
+        return 1;
+    }
     const long long n_tiles = (long long)((N + NT - 1) / NT) * ((M + GT - 1) / GT);
     const long long resident = (long long)n_sm * (wide ? GemmCfg<256>::CTAS : GemmCfg<128>::CTAS);
     const unsigned grid = (unsigned)(n_tiles < resident ? n_tiles : resident);
