@@ -15,6 +15,8 @@
 // by commits, warps 2-5 read an accumulator when its last commit arrives, hand it back as soon as
 // it is in registers, and either store bf16 rows or add into an fp32 C (tiles of one launch are
 // disjoint and launches on a stream are ordered, so the addition is a plain load-add-store).
+#include <cstdint>
+
 #include "peagle_internal.h"
 #include "sm100_ptx.cuh"
 
@@ -255,12 +257,16 @@ struct Gemm2Cfg {
     static constexpr int STAGE_BYTES = 2 * G_TILE_BYTES; // A: 128 m x 64 k, B half: 128 n x 64 k
     static constexpr int OFF_BAR = STAGES * STAGE_BYTES;
     static constexpr int N_BAR = 2 * STAGES + 4; // full, empty per stage; accumulator full / empty x 2
-    static constexpr int SMEM = OFF_BAR + N_BAR * 8 + 32 + 1024;
+    // two 128 x 32 fp32 tiles through which an accumulate-mode C leaves by tiled reduce-adds
+    static constexpr int OFF_OUT = OFF_BAR + 1024;
+    static constexpr int OUT_BYTES = GT * 32 * 4;
+    static constexpr int SMEM = OFF_OUT + 2 * OUT_BYTES + 1024;
+    static_assert(N_BAR * 8 + 32 <= 1024 && SMEM <= 227 * 1024, "shared memory of one CTA");
 };
 
 __global__ void __launch_bounds__(192, 1)
 gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-             const GemmParams P)
+             const __grid_constant__ CUtensorMap tmC, const GemmParams P)
 {
     using C = Gemm2Cfg;
     constexpr int NT = C::NT, ST = C::STAGES;
@@ -376,12 +382,13 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
     } else {
         // ------------------------------------------------------------ epilogue (warps 2-5, each CTA)
         const int q = warp & 3;
-        int j = 0;
+        int j = 0, piece = 0;
         for (int t = pair; t < n_tiles; t += n_pairs, ++j) {
             const int buf = j & 1;
             const int m = (t / tiles_n) * 2 * GT + (int)rank * GT + q * 32 + lane;
             const int n0 = (t % tiles_n) * NT;
-            if (!__all_sync(0xffffffffu, mbar_wait_cluster(ACCFULL(buf), (j >> 1) & 1, abort_flag)))
+            // the four warps go on, or leave, together (they meet at named barriers below)
+            if (!bar_and(2, 128, mbar_wait_cluster(ACCFULL(buf), (j >> 1) & 1, abort_flag)))
                 break;
             tc_fence_after();
             const uint32_t trow = tmem + ((uint32_t)(q * 32) << 16) + buf * NT;
@@ -397,6 +404,33 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                         mbar_arrive_remote(ACCEMPTY(buf), 0);
                 }
                 const int n = n0 + c * 32;
+                if (P.c_f32_add) {
+                    // fp32 C: the 128 x 32 piece goes through a swizzled tile in shared memory and
+                    // is added to C by one tiled reduce-add (whole 128-byte rows reach L2 together;
+                    // rows and columns past the matrix are clipped by the tensor map).  Two tiles
+                    // alternate: a tile is rewritten once the reduce-add issued two pieces ago has
+                    // read it.
+                    const uint32_t ob = sb + C::OFF_OUT + (uint32_t)(piece & 1) * C::OUT_BYTES;
+                    if (threadIdx.x == 64)
+                        bulk_wait_group_read<1>();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int rw = q * 32 + lane;
+                    uint8_t *dst = sp + C::OFF_OUT + (piece & 1) * C::OUT_BYTES + rw * 128;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        *reinterpret_cast<uint4 *>(dst + ((i ^ (rw & 7)) << 4)) =
+                            make_uint4(o[4 * i], o[4 * i + 1], o[4 * i + 2], o[4 * i + 3]);
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (threadIdx.x == 64) {
+                        const int row0 = (t / tiles_n) * 2 * GT + (int)rank * GT;
+                        if (n < P.N && row0 < P.M) // a piece wholly outside C is not sent at all
+                            tma_reduce_add_2d(&tmC, ob, n, row0);
+                        bulk_commit_group();
+                    }
+                    ++piece;
+                    continue;
+                }
                 if (m >= P.M)
                     continue;
                 if (!P.c_f32_add) {
@@ -412,22 +446,11 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                             *reinterpret_cast<uint4 *>(dst + i) = v;
                         }
                     }
-                } else {
-                    float *dst = static_cast<float *>(P.C) + (size_t)m * P.ldc + n;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        if (n + i < P.N) {
-                            float4 v = *reinterpret_cast<float4 *>(dst + i);
-                            v.x += __uint_as_float(o[i + 0]);
-                            v.y += __uint_as_float(o[i + 1]);
-                            v.z += __uint_as_float(o[i + 2]);
-                            v.w += __uint_as_float(o[i + 3]);
-                            *reinterpret_cast<float4 *>(dst + i) = v;
-                        }
-                    }
                 }
             }
         }
+        if (threadIdx.x == 64)
+            bulk_wait_group<0>(); // the last reduce-adds have left shared memory and reached C
     }
 
     // ------------------------------------------------------------ teardown
@@ -523,7 +546,21 @@ int launch_gemm(EncodeTiledFn enc, const void *A, long long lda, int a_t, const 
         const long long tiles2 = (long long)((N + 255) / 256) * ((M + 255) / 256);
         const long long n_pairs = tiles2 < fit ? tiles2 : fit;
         cfg.gridDim = dim3((unsigned)(2 * n_pairs));
-        if (cudaLaunchKernelEx(&cfg, gemm2_kernel, tmA, tmB, P) != cudaSuccess)
+        // fp32 C as a tensor for the tiled reduce-adds: 32 columns (128 bytes) x 128 rows
+        CUtensorMap tmC = tmA;
+        if (c_f32_add) {
+            if (reinterpret_cast<uintptr_t>(C) & 15)
+                return PEAGLE_ERR_ALIGN;
+            cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+            cuuint64_t strides[1] = {(cuuint64_t)ldc * 4};
+            cuuint32_t box[2] = {32, (cuuint32_t)GT};
+            cuuint32_t estr[2] = {1, 1};
+            if (enc(&tmC, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return PEAGLE_ERR_CUDA;
+        }
+        if (cudaLaunchKernelEx(&cfg, gemm2_kernel, tmA, tmB, tmC, P) != cudaSuccess)
             return PEAGLE_ERR_CUDA;
         return 1;
     }

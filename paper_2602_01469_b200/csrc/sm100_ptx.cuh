@@ -167,6 +167,15 @@ __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap *m, uint32_t
         "r"(src), "r"(x), "r"(y), "r"(z)
         : "memory");
 }
+// The same for a 2-D tensor map.
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap *m, uint32_t src, int x, int y)
+{
+    asm volatile(
+        "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+            reinterpret_cast<uint64_t>(m)),
+        "r"(src), "r"(x), "r"(y)
+        : "memory");
+}
 // Bulk reduce-add of fp32 from shared to global memory (both 16-byte aligned, size % 16 == 0).
 __device__ __forceinline__ void bulk_reduce_add_f32(void *gdst, uint32_t ssrc, uint32_t bytes)
 {
