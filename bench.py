@@ -502,6 +502,71 @@ def run_gemm(args, w):
     ctx.close()
 
 
+def run_layer(args, w):
+    """The layer slice as Section 3.2 trains it: per segment the fused projection (its own rows and
+    the depth-0 rows it sees, projected again), the rotary prologue, masked attention forward and
+    backward, and the gradients back through the projection into dX / dW.  A side line: time per
+    pass and the useful work of its attention and projection parts."""
+    import torch
+
+    from paper_2602_01469_b200 import binding
+
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = binding.Context(0)
+    cu, anchor, depth, parts = inputs.build_case(w, binding.peagle_assign_segments)
+    T, dm = int(cu[-1]), args.d_model
+    nqkv = (w.n_q_heads + 2 * w.n_kv_heads) * w.head_dim
+    X, W, dO = (t.to(dev) for t in inputs.make_layer_tensors(T, dm, w.n_q_heads, w.n_kv_heads, w.head_dim, w.seed))
+    prob = binding.Problem(cu, torch.from_numpy(anchor).to(dev), torch.from_numpy(depth).to(dev), w.K,
+                           w.n_q_heads, w.n_kv_heads, w.head_dim, w.scale)
+    bparts = [binding.Partition(p["seq"], p["q"], p["k"]) for p in parts]
+    O = torch.empty(T, w.n_q_heads, w.head_dim, dtype=torch.bfloat16, device=dev)
+    LSE = torch.empty(w.n_q_heads, T, dtype=torch.float32, device=dev)
+    dX = torch.empty(T, dm, dtype=torch.bfloat16, device=dev)
+    dW = torch.empty(nqkv, dm, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step():
+        binding.peagle_layer_partitioned(ctx, prob, bparts, X, W, 10000.0, dO, O, LSE, dX, dW, stream)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert binding.peagle_poll_status(ctx) == 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(0) as clocks:
+        torch.cuda.synchronize()
+        e0.record(stream)
+        for _ in range(args.steps):
+            step()
+        e1.record(stream)
+        torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    # rows projected per pass: every segment's own rows with all heads (forward, dX, dW: three
+    # products over the fused width) and the earlier depth-0 rows it sees with the K / V heads only
+    own = sum(p["q"][1] - p["q"][0] for p in parts)
+    seen = sum(sum(e - b for b, e in p["k"]) for p in parts) - own
+    kvw = 2 * w.n_kv_heads * w.head_dim
+    f_gemm = 3 * 2.0 * dm * (own * nqkv + seen * kvw)
+    f_fwd, f_bwd = useful_flops(w)
+    peaks, src = load_peaks()
+    peak = float(peaks["bf16_tflops"])
+    tf = (f_gemm + f_fwd + f_bwd) / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "layer slice (projection, rotary, masked attention; forward+backward per segment) useful TFLOP/s",
+        "value": tf, "unit": UNIT, "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "rows": T, "segments": len(parts), "d_model": dm, "fused_width": nqkv,
+                   "rows_projected_again": int(seen), "attention_tflop": (f_fwd + f_bwd) / 1e12,
+                   "projection_tflop": f_gemm / 1e12, "l2": "tensors larger than L2, no flush"},
+        "clocks": clocks.summary(),
+        "roofline": {"kernel": "whole pass", "bound": "tensor", "achieved": tf, "peak": peak, "unit": UNIT,
+                     "frac": tf / peak, "traffic": None, "peak_source": "%s bf16_tflops (burst)" % src},
+    }))
+    ctx.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -509,10 +574,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=inputs.HEADLINE, choices=sorted(inputs.WORKLOADS))
-    ap.add_argument("--op", default="attention", choices=["attention", "rope", "gemm"],
+    ap.add_argument("--op", default="attention", choices=["attention", "rope", "gemm", "layer"],
                     help="attention: the hot path (default); rope: the rotary prologue side line; "
-                         "gemm: the layer slice's projection products side line")
-    ap.add_argument("--d-model", type=int, default=2880, help="hidden width for --op gemm")
+                         "gemm: the layer slice's projection products side line; layer: the whole layer slice, "
+                         "segment by segment")
+    ap.add_argument("--d-model", type=int, default=2880, help="hidden width for --op gemm / layer")
     ap.add_argument("--parallelism", default="replicas", choices=["replicas", "partitions"],
                     help="with --gpus N > 1: N independent replicas of the workload (default), or one "
                          "workload whose query partitions are dealt out over the ranks (dK / dV "
@@ -528,6 +594,8 @@ def main():
         run_rope(args, w)
     elif args.op == "gemm":
         run_gemm(args, w)
+    elif args.op == "layer":
+        run_layer(args, w)
     else:
         run_cuda(args, w)
 
