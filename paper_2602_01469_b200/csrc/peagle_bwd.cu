@@ -296,8 +296,10 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (was_last && wk.valid)
                     ok = load_kv(wk.w, wk.kt, wk.g); // next item's K / V into the other stage
             }
-        } else if (warp == 8 && lane == 0) {
-            // -------------------------------------------------------- MMA issue
+        } else if (warp == 8) {
+            // -------------------------------------------------------- MMA issue: the whole warp
+            // walks the steps and waits, its elected lane issues (see elect_one)
+            const uint32_t lead = elect_one();
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
             constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
             constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
@@ -315,12 +317,12 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             auto issue_s = [&](uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ts_lo(tmem + C::TM_S, tmem + C::TM_K + k * 8, q_k + q + k * 2, IDESC_S, k > 0);
+                    if (lead) mma_ts_lo(tmem + C::TM_S, tmem + C::TM_K + k * 8, q_k + q + k * 2, IDESC_S, k > 0);
             };
             auto issue_dp = [&](uint32_t q) {
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ts_lo(tmem + C::TM_DP, tmem + C::TM_V + k * 8, q_k + q + TBU + k * 2, IDESC_S,
+                    if (lead) mma_ts_lo(tmem + C::TM_DP, tmem + C::TM_V + k * 8, q_k + q + TBU + k * 2, IDESC_S,
                               k > 0);
             };
             // The issuing thread is a serial instruction stream, so it keeps its bookkeeping
@@ -345,9 +347,9 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     break;
                 tc_fence_after();
                 issue_s((it % 3) * 2 * TBU);
-                tc_commit(BAR(B_SFULL));
+                if (lead) tc_commit(BAR(B_SFULL));
                 issue_dp((it % 3) * 2 * TBU);
-                tc_commit(BAR(B_DPFULL));
+                if (lead) tc_commit(BAR(B_DPFULL));
                 for (int i = 0; ok && i < n_cur; ++i, ++it) {
                     const int st = it % 3, nst = (it + 1) % 3;
                     const uint32_t qo = st * 2 * TBU, nqo = nst * 2 * TBU;
@@ -361,7 +363,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                        if (lead) mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + TBU + k * 128, IDESC_KV, !first || k > 0);
                     if (!last) {
                         ok = mbar_wait(BAR(B_QFULL + nst), ((it + 1) / 3) & 1, abort_flag);
@@ -369,7 +371,7 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                             break;
                         tc_fence_after();
                         issue_s(nqo);
-                        tc_commit(BAR(B_SFULL));
+                        if (lead) tc_commit(BAR(B_SFULL));
                     }
                     // ---- dK(it), dQ(it) once dS^T(it) is in tensor and shared memory, then
                     // dP^T(it+1); the single dQ accumulator must have been read out
@@ -380,19 +382,19 @@ bwd64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ts_lo(tmem + C::TM_DK, tmem + C::TM_DP + (k / 4) * 64 + (k % 4) * 8,
+                        if (lead) mma_ts_lo(tmem + C::TM_DK, tmem + C::TM_DP + (k / 4) * 64 + (k % 4) * 8,
                                   q_m + qo + k * 128, IDESC_KV, !first || k > 0);
-                    tc_commit(BAR(B_QEMPTY + st)); // dQ reads neither Q nor dO
+                    if (lead) tc_commit(BAR(B_QEMPTY + st)); // dQ reads neither Q nor dO
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, kv_m + kvo + k * 128, IDESC_DQ,
+                        if (lead) mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, kv_m + kvo + k * 128, IDESC_DQ,
                                   k > 0);
-                    tc_commit(BAR(B_DQFULL));
-                    if (last)
-                        tc_commit(BAR(B_KVEMPTY + ks));
-                    else {
+                    if (lead) tc_commit(BAR(B_DQFULL));
+                    if (last) {
+                        if (lead) tc_commit(BAR(B_KVEMPTY + ks));
+                    } else {
                         issue_dp(nqo);
-                        tc_commit(BAR(B_DPFULL));
+                        if (lead) tc_commit(BAR(B_DPFULL));
                     }
                 }
                 if (!ok)

@@ -295,8 +295,10 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                 if (was_last && wk.valid)
                     ok = load_kv(wk.w, wk.kt, wk.g);
             }
-        } else if (warp == 8 && lane == 0) {
-            // -------------------------------------------------------- MMA issue
+        } else if (warp == 8) {
+            // -------------------------------------------------------- MMA issue: the whole warp
+            // walks the steps and waits, its elected lane issues (see elect_one)
+            const uint32_t lead = elect_one();
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, 128, 0, 0);
             constexpr uint32_t IDESC_KV = idesc_bf16_f32(128, D, 0, 1);
             constexpr uint32_t IDESC_DQ = idesc_bf16_f32(128, D, 1, 1);
@@ -313,12 +315,12 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
             auto issue_s = [&](uint32_t q) { // S^T = K Q^T
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss_lo(tmem + C::TM_S, k_k + koff(k), q_k + q + koff(k), IDESC_S, k > 0);
+                    if (lead) mma_ss_lo(tmem + C::TM_S, k_k + koff(k), q_k + q + koff(k), IDESC_S, k > 0);
             };
             auto issue_dp = [&]() { // dP^T = V dO^T
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k)
-                    mma_ss_lo(tmem + C::TM_DP, v_k + koff(k), do_k + koff(k), IDESC_S, k > 0);
+                    if (lead) mma_ss_lo(tmem + C::TM_DP, v_k + koff(k), do_k + koff(k), IDESC_S, k > 0);
             };
             const int G = P.Hq / P.Hkv;
             bool ok = true;
@@ -340,9 +342,9 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                     break;
                 tc_fence_after();
                 issue_s((it & 1) * TBU);
-                tc_commit(BAR(B_SFULL));
+                if (lead) tc_commit(BAR(B_SFULL));
                 issue_dp();
-                tc_commit(BAR(B_DPFULL));
+                if (lead) tc_commit(BAR(B_DPFULL));
                 for (int i = 0; ok && i < n_cur; ++i, ++it) {
                     const int st = it & 1, nst = st ^ 1;
                     static_assert(NSQ == 2, "stage = step parity");
@@ -357,16 +359,16 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k) // query rows 16k..16k+15 of P^T (bf16 over S^T)
-                        mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
+                        if (lead) mma_ts_lo(tmem + C::TM_DV, tmem + C::TM_S + (k / 4) * 64 + (k % 4) * 8,
                                   do_m + k * 128, IDESC_KV, !first || k > 0);
-                    tc_commit(BAR(B_DOEMPTY)); // dV is the step's last product with dO
+                    if (lead) tc_commit(BAR(B_DOEMPTY)); // dV is the step's last product with dO
                     if (!last) {
                         ok = mbar_wait(BAR(B_QFULL + nst), ((it + 1) >> 1) & 1, abort_flag);
                         if (!ok)
                             break;
                         tc_fence_after();
                         issue_s(nqo);
-                        tc_commit(BAR(B_SFULL));
+                        if (lead) tc_commit(BAR(B_SFULL));
                     }
                     // ---- dK(it), dQ(it) once dS^T(it) is in shared memory (the compute warps then
                     // hold dP^T(it) in registers: dQ goes over its columns)
@@ -376,15 +378,15 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                     tc_fence_after();
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ss_lo(tmem + C::TM_DK, ds_k + koff(k), q_m + qo + k * 128, IDESC_KV,
+                        if (lead) mma_ss_lo(tmem + C::TM_DK, ds_k + koff(k), q_m + qo + k * 128, IDESC_KV,
                                   !first || k > 0);
-                    tc_commit(BAR(B_QEMPTY + st)); // dQ reads neither Q nor dO
+                    if (lead) tc_commit(BAR(B_QEMPTY + st)); // dQ reads neither Q nor dO
 #pragma unroll
                     for (int k = 0; k < 8; ++k)
-                        mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, k_m + k * 128, IDESC_DQ, k > 0);
-                    tc_commit(BAR(B_DQFULL));
+                        if (lead) mma_ss_lo(tmem + C::TM_DQ, ds_m + k * 128, k_m + k * 128, IDESC_DQ, k > 0);
+                    if (lead) tc_commit(BAR(B_DQFULL));
                     if (last) {
-                        tc_commit(BAR(B_KVEMPTY));
+                        if (lead) tc_commit(BAR(B_KVEMPTY));
                     } else {
                         // ---- dP^T(it+1) over the columns dQ(it) has just left
                         ok = mbar_wait(BAR(B_DQEMPTY), it & 1, abort_flag) &&
@@ -393,7 +395,7 @@ bwd128_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ C
                             break;
                         tc_fence_after();
                         issue_dp();
-                        tc_commit(BAR(B_DPFULL));
+                        if (lead) tc_commit(BAR(B_DPFULL));
                     }
                 }
                 if (!ok)

@@ -320,7 +320,9 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // tiles are independent instruction streams (they only share the K / V stages, which are
         // released once both threads have committed), and two threads issue twice as fast as one.
         const int x = (warp - 8) >> 1;
-        if (lane == 0 && x < ntile) {
+        // the whole warp walks the items and waits, its elected lane issues (see elect_one)
+        const uint32_t lead = elect_one();
+        if (x < ntile) {
             constexpr uint32_t IDESC_S = idesc_bf16_f32(128, BN, 0, 0);
             constexpr uint32_t IDESC_O = idesc_bf16_f32(128, D, 0, 1);
             constexpr uint32_t TU = C::TILE_BYTES >> 4, PU = C::PANEL_BYTES >> 4;
@@ -335,19 +337,19 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 #pragma unroll
                 for (int k = 0; k < D / 16; ++k) {
                     const uint32_t off = (k / 4) * PU + (k % 4) * 2;
-                    mma_ss_lo(tS, q_lo + off, kb + off, IDESC_S, k > 0);
+                    if (lead) mma_ss_lo(tS, q_lo + off, kb + off, IDESC_S, k > 0);
                 }
-                tc_commit(BAR(B_SFULL + x));
-                tc_commit(BAR(B_KEMPTY + st));
+                if (lead) tc_commit(BAR(B_SFULL + x));
+                if (lead) tc_commit(BAR(B_KEMPTY + st));
             };
             auto issue_pv = [&](int st, bool acc) {
                 const uint32_t vb = v_lo + st * TU;
-                mma_ts_lo(tO, tP, vb, IDESC_O, acc);
+                if (lead) mma_ts_lo(tO, tP, vb, IDESC_O, acc);
 #pragma unroll
                 for (int k = 1; k < BN / 16; ++k)
-                    mma_ts_lo(tO, tP + k * 8, vb + k * 128, IDESC_O, 1);
-                tc_commit(BAR(B_PVDONE + x));
-                tc_commit(BAR(B_VEMPTY + st));
+                    if (lead) mma_ts_lo(tO, tP + k * 8, vb + k * 128, IDESC_O, 1);
+                if (lead) tc_commit(BAR(B_PVDONE + x));
+                if (lead) tc_commit(BAR(B_VEMPTY + st));
             };
             uint32_t kpos = 0; // position in the K / V ring, running over the items
             uint32_t t = 0;    // key tiles of this thread's tile so far (phases of S, P, PV)
@@ -368,7 +370,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                          mbar_wait(BAR(B_VFULL + pos % NS), (pos / NS) & 1, abort_flag);
                 }
                 if (ok && cnt == 0)
-                    mbar_arrive(BAR(B_QEMPTY)); // no product reads this Q
+                    if (lead) mbar_arrive(BAR(B_QEMPTY)); // no product reads this Q
                 if (ok && cnt > 0) {
                     const uint32_t p0 = kpos + n_single;
                     // S of the previous item's last key tile must be in the softmax registers
@@ -378,7 +380,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                         tc_fence_after();
                         issue_s(p0 % NS);
                         if (cnt == 1)
-                            tc_commit(BAR(B_QEMPTY));
+                            if (lead) tc_commit(BAR(B_QEMPTY));
                     }
                 }
                 for (int j = 0; ok && j < cnt; ++j) {
@@ -396,7 +398,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                             tc_fence_after();
                             issue_s(nst);
                             if (j + 2 == cnt)
-                                tc_commit(BAR(B_QEMPTY)); // the item's last product with Q
+                                if (lead) tc_commit(BAR(B_QEMPTY)); // the item's last product with Q
                         }
                     }
                     ok = mbar_wait(BAR(B_VFULL + st), ph, abort_flag) &&
@@ -413,7 +415,7 @@ fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                                 break;
                             issue_s(nst);
                             if (j + 2 == cnt)
-                                tc_commit(BAR(B_QEMPTY));
+                                if (lead) tc_commit(BAR(B_QEMPTY));
                         }
                     }
                 }

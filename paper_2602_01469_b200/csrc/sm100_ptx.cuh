@@ -426,6 +426,21 @@ __device__ __forceinline__ void mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint
         : "memory");
 }
 
+// One lane of the (converged) calling warp gets 1, the others 0.  A warp that issues tcgen05
+// products should stay converged, pick its issuing lane with this instruction once, and guard only
+// the product and commit statements with the result: the compiler then keeps the descriptors and
+// addresses, which are the same in every lane, in uniform registers, where the instruction reads
+// its operands.  A lone thread in a `lane == 0` branch computes them in ordinary registers and
+// moves every word across for every product (about nine moves per product): measured, the
+// products of a step then issue at 103 clocks each beside arithmetic-heavy warps, against 65 this
+// way (the tensor pipe's own rate).
+__device__ __forceinline__ uint32_t elect_one()
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(r));
+    return r;
+}
+
 // The same for a whole, converged warp: every lane carries the (warp-uniform) operands and only
 // the lane with `lead` != 0 issues.  Keeping the issuing warp converged lets the compiler do the
 // descriptor arithmetic once per warp in the uniform datapath, where the instruction wants its
