@@ -135,8 +135,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issue
-        if (lane == 0) {
+        // ------------------------------------------------------------ MMA issue (whole warp
+        // converged, elected lane issues: see elect_one)
+        const uint32_t lead = elect_one();
+        {
             const uint32_t idesc = idesc_bf16_f32(GT, NT, P.a_t, P.b_t);
             // K-major: a k = 16 slice is 32 bytes further inside the 128-byte rows; MN-major: 16
             // rows (2,048 bytes) further, the second 64-wide panel half a tile on
@@ -161,12 +163,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUt
                 const uint32_t b_lo = desc_lo_sw128(b, P.b_t ? G_TILE_BYTES / 2 : 16);
 #pragma unroll
                 for (int k = 0; k < GK / 16; ++k)
-                    mma_ss_lo(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
+                    if (lead) mma_ss_lo(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
                               (i > 0 || k > 0) ? 1u : 0u);
-                tc_commit(EMPTY(s));
+                if (lead) tc_commit(EMPTY(s));
             }
             if (ok)
-                tc_commit(ACCFULL(buf));
+                if (lead) tc_commit(ACCFULL(buf));
             }
         }
     } else {
@@ -348,8 +350,10 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
             }
         }
     } else if (warp == 1) {
-        if (lane == 0 && rank == 0) {
-            // ---------------------------------------- first CTA: the pair's products
+        const uint32_t lead = elect_one();
+        if (rank == 0) {
+            // ---------------------------------------- first CTA: the pair's products (whole warp
+            // converged, elected lane issues: see elect_one)
             const uint32_t idesc = idesc_bf16_f32(2 * GT, NT, P.a_t, P.b_t);
             const uint32_t a_step = P.a_t ? 128u : 2u, b_step = P.b_t ? 128u : 2u;
             bool ok = true;
@@ -371,12 +375,12 @@ gemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CU
                     const uint32_t b_lo = desc_lo_sw128(b, P.b_t ? G_TILE_BYTES / 2 : 16);
 #pragma unroll
                     for (int k = 0; k < GK / 16; ++k)
-                        mma_ss_lo_pair(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
+                        if (lead) mma_ss_lo_pair(tmem + buf * NT, a_lo + k * a_step, b_lo + k * b_step, idesc,
                                        (i > 0 || k > 0) ? 1u : 0u);
-                    tc_commit_pair(EMPTY(s));
+                    if (lead) tc_commit_pair(EMPTY(s));
                 }
                 if (ok)
-                    tc_commit_pair(ACCFULL(buf));
+                    if (lead) tc_commit_pair(ACCFULL(buf));
             }
         }
     } else {
