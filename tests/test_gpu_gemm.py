@@ -23,7 +23,8 @@ def rand_bf16(shape, seed):
 
 
 @pytest.mark.parametrize("M,N,K", [(128, 128, 64), (200, 264, 200), (1, 8, 8), (513, 1024, 2880), (300, 72, 1000),
-                                   (300, 1160, 520)])  # the last: wide tiles with a ragged last column of tiles
+                                   (300, 1160, 520),   # wide tiles with a ragged last column of tiles
+                                   (200, 1024, 136)])  # one pair of CTAs whose second CTA holds 72 rows
 @pytest.mark.parametrize("a_t,b_t", [(0, 0), (0, 1), (1, 1), (1, 0)])
 def test_products_match_fp64(ctx, M, N, K, a_t, b_t):
     def pad8(x):
