@@ -11,7 +11,11 @@ namespace peagle {
 constexpr int BM = 128;          // query rows per tile
 constexpr int BN = 128;          // keys per tile
 constexpr int MAX_KRANGES = 32;  // visible key ranges per partition
-constexpr int BWD_CQ = 4;        // query tiles per backward work item (aligned chunk; at most 8)
+#ifndef PEAGLE_BWD_CQ
+#define PEAGLE_BWD_CQ 4 // measured: 2 / 4 / 8 give 3.33 / 3.27 / 3.38 ms for the head_dim 64 main kernel
+#endif
+constexpr int BWD_CQ = PEAGLE_BWD_CQ; // query tiles per backward work item (aligned chunk; at most 8)
+static_assert(BWD_CQ >= 1 && BWD_CQ <= 8, "the chunk's mask word has eight bits per field");
 constexpr int32_t META_NONE_Q = -1;         // packed metadata of a row outside the partition (sees nothing)
 constexpr int32_t META_NONE_K = 0x7fffffff; // packed metadata of a key outside the batch (seen by nobody)
 
